@@ -1,0 +1,192 @@
+/*
+ * amph.h - C ABI of the B200 (sm_100a) Amphista speculative-decoding step.
+ *
+ * One decoding step of Amphista (arXiv 2406.13170) for a Llama/Vicuna-shaped target at
+ * batch 1:  draft module (Section 3, Eq. 1-6)  ->  candidate tree (Appendix A.1)  ->
+ * target forward over all tree tokens under a tree-causal mask (Section 2 "Tree
+ * Attention", Fig. 5)  ->  greedy longest-prefix acceptance and KV-cache compaction
+ * (Section 2 "Speculative Decoding", Section 3.2 last paragraph).
+ *
+ * Conventions
+ *   - Every function returns an amph_status; none throws, aborts or exits.
+ *     amph_last_error() gives a human-readable message for the last failure on a context.
+ *   - OWNERSHIP: the caller allocates and owns all device memory (weights, the KV region,
+ *     the workspace) and passes raw device pointers; they must stay valid and unmoved
+ *     until amph_destroy.  The library owns only the host-side amph_ctx.  The library
+ *     never allocates device memory.
+ *   - All device work is enqueued on the stream given to amph_init (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream).
+ *   - Pointers documented "host or device" may be pageable/pinned host memory or device
+ *     memory; results are copied with a stream-ordered copy and are valid once the
+ *     caller has synchronised the stream.  Pointers documented "host" are read or written
+ *     before the call returns.
+ *   - Linear weights are row-major [out_features, in_features]; vectors are contiguous.
+ *   - Requires an sm_100a device.  There is no CPU path: without the device every call
+ *     that needs one fails with AMPH_ERR_CUDA.
+ */
+#ifndef AMPH_H_
+#define AMPH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t amph_status;
+enum {
+  AMPH_OK = 0,
+  AMPH_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, unknown name            */
+  AMPH_ERR_SHAPE = 2,          /* unsupported model / tree shape, tensor shape mismatch     */
+  AMPH_ERR_STATE = 3,          /* call order violated (see the state machine below)         */
+  AMPH_ERR_CAPACITY = 4,       /* ctx_len + tree nodes would exceed max_ctx                 */
+  AMPH_ERR_WORKSPACE = 5,      /* kv / workspace region too small or misaligned             */
+  AMPH_ERR_MISSING_WEIGHT = 6, /* amph_load_weights did not receive every tensor           */
+  AMPH_ERR_CUDA = 7,           /* a CUDA runtime / driver call failed                       */
+  AMPH_ERR_TIMEOUT = 8         /* a bounded device-side wait gave up (pipeline barrier)     */
+};
+
+enum { AMPH_DTYPE_F32 = 0, AMPH_DTYPE_BF16 = 1 };
+
+/* amph_config.flags */
+enum {
+  AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
+  AMPH_FLAG_NO_GRAPH = 2        /* launch kernels one by one instead of replaying a CUDA graph */
+};
+
+#define AMPH_MAX_HEADS_K 8
+#define AMPH_MAX_NODES 128
+#define AMPH_TOPK_STRIDE 16
+
+typedef struct amph_ctx amph_ctx;
+
+/* Shapes of the target model and of the draft module.
+ * Target: Llama architecture (RMSNorm, rotary embedding on pairs (i, i + head_dim/2),
+ * multi-head attention with n_heads * head_dim == d_model, SwiGLU FFN, untied lm_head).
+ * Draft module (Section 3): n_sal staged adaptation layers, each one decoder layer of the
+ * target's shape with its own KV cache and a preceding fc: 2d -> d; K head MLPs d -> d;
+ * positional embedding PE [K, d]; aeb_layers unmasked self-attention layers with n_heads
+ * heads; K vocabulary projections [vocab, d]; head k keeps its top topk[k] candidates. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t weight_dtype;   /* AMPH_DTYPE_*: storage type of every weight tensor             */
+  int32_t kv_dtype;       /* AMPH_DTYPE_*: storage type of all KV caches (must equal weight_dtype) */
+  int32_t max_ctx;        /* KV capacity in slots (committed tokens + tree nodes)           */
+  int32_t max_batch;      /* must be 1                                                      */
+  int32_t K;              /* drafting heads, 1..AMPH_MAX_HEADS_K (the paper uses 4)         */
+  int32_t n_sal;          /* staged adaptation layers: 2 (the paper's design) or 1          */
+  int32_t aeb_layers;     /* 1 (the paper's design) or 2 (its "alpha" variant)              */
+  int32_t topk[AMPH_MAX_HEADS_K]; /* candidates kept per head, each 1..AMPH_TOPK_STRIDE     */
+  int32_t flags;          /* AMPH_FLAG_*                                                    */
+} amph_config;
+
+/* Draft-tree topology (Appendix A.1): node 0 is the root (the token the target chose last);
+ * a node of depth k >= 1 carries head k's candidate of rank `rank`.  Nodes must be sorted so
+ * that parent[n] < n.  All three arrays are HOST pointers of n_nodes entries, copied by
+ * amph_init.  n_nodes <= AMPH_MAX_NODES; depth <= K; rank[n] < topk[depth[n]-1]. */
+typedef struct {
+  int32_t n_nodes;
+  const int16_t* parent;  /* parent[0] = -1 */
+  const uint8_t* depth;   /* depth[0] = 0   */
+  const uint8_t* rank;    /* rank[0] ignored */
+} amph_tree;
+
+/* One named weight tensor in device memory (borrowed, not copied). */
+typedef struct {
+  const char* name;
+  const void* dev_ptr;    /* 16-byte aligned, contiguous row-major */
+  int32_t dtype;          /* AMPH_DTYPE_*, must equal config.weight_dtype */
+  int32_t ndim;           /* 1 or 2 */
+  int64_t shape[4];
+} amph_tensor;
+
+/* State machine: amph_init -> amph_load_weights -> amph_prefill ->
+ *   ( amph_draft -> amph_verify_tree -> amph_accept )*   or   amph_step*
+ * A call out of order returns AMPH_ERR_STATE and changes nothing. */
+
+/* Sizes of the two device regions the caller must provide for (config, tree).
+ * kv_bytes: target KV cache + the adaptation layers' KV caches; ws_bytes: activations,
+ * partial sums, state.  Host-only computation; no device needed. */
+amph_status amph_workspace_bytes(const amph_config* cfg, const amph_tree* tree,
+                                 size_t* kv_bytes, size_t* ws_bytes);
+
+/* Creates a context.  kv_dev / ws_dev: device regions of at least the sizes above, 256-byte
+ * aligned, owned by the caller.  Validates shapes, builds the tree tables (ancestor bitmasks,
+ * positions: Fig. 5) and zeroes the state.  stream: cudaStream_t as void*. */
+amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_dev, size_t kv_bytes,
+                      void* ws_dev, size_t ws_bytes, void* stream, amph_ctx** out);
+
+/* Registers the weights.  Names (i = layer, s = 1..n_sal, k = 0..K-1, l = 0..aeb_layers-1):
+ *   tok_emb [V,d]; layers.{i}.{attn_norm [d], wq, wk, wv, wo [d,d], ffn_norm [d],
+ *   w_gate, w_up [F,d], w_down [d,F]}; final_norm [d]; lm_head [V,d];
+ *   draft.fc{s} [d,2d] (Eq. 1; input order [hidden ; token embedding]);
+ *   draft.sal{s}.<the nine per-layer names>; draft.mlp.{k}.w [d,d], draft.mlp.{k}.b [d] (Eq. 2);
+ *   draft.pe [K,d] (Eq. 4); draft.aeb.{l}.{wq,wk,wv,wo} [d,d] (Eq. 5); draft.lm_head.{k} [V,d] (Eq. 6).
+ * May be called several times; AMPH_ERR_MISSING_WEIGHT is reported by amph_prefill if a tensor
+ * was never given.  Pointers are borrowed. */
+amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t n);
+
+/* Causal forward of the prompt through the target (fills its KV cache), greedy choice of the
+ * root token, and the adaptation layers over all prompt positions but the last, which stays
+ * pending for the first draft (Eq. 1: their caches cover positions before t).
+ * prompt_ids: HOST, n >= 1 ids in [0, vocab).  out_root: HOST, may be NULL.  Synchronises the
+ * stream before returning.  Resets any previous sequence. */
+amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, int32_t* out_root);
+
+/* Draft module (Section 3): adaptation layers over the pending rows (Eq. 1), K head MLPs on
+ * the last row (Eq. 2), + PE (Eq. 3-4), bi-directional self-attention across the K rows (Eq. 5),
+ * K vocabulary projections and top-k (Eq. 6), then tree tokens (Appendix A.1).
+ * out_topk_ids [K][AMPH_TOPK_STRIDE] int32, out_topk_vals [K][AMPH_TOPK_STRIDE] float: host or
+ * device, may be NULL; row k holds topk[k] entries ordered by value descending, equal values by
+ * ascending id. */
+amph_status amph_draft(amph_ctx* ctx, int32_t* out_topk_ids, float* out_topk_vals);
+
+/* Target forward over the n_nodes tree tokens (Section 2, Fig. 5): node n at position
+ * ctx_len + depth[n], its key / value in slot ctx_len + n, attending the ctx_len committed
+ * slots and its ancestors.  tree_tokens: host or device [n_nodes] int32, or NULL to use the
+ * tokens amph_draft built; entries < 0 keep the drafted token, entry 0 is always the root.
+ * out_argmax: host or device [n_nodes] int32 (greedy choice after each node; ties -> lowest id),
+ * may be NULL. */
+amph_status amph_verify_tree(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_argmax);
+
+/* Greedy acceptance (Section 2): the deepest root path on which every drafted token equals the
+ * target's greedy choice at its parent; compacts the accepted nodes' key / value rows to slots
+ * ctx_len .. ctx_len + n - 1, advances ctx_len by n, and queues the accepted rows for the next draft.
+ * out_tokens [K+1], out_n [1], out_path [K+1] (node ids), out_next_root [1]: host or device int32,
+ * each may be NULL. */
+amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_t* out_path,
+                        int32_t* out_next_root);
+
+/* draft -> tree -> verify -> accept, enqueued back to back with no host synchronisation.
+ * out_tokens [K+1], out_n [1]: host or device int32, may be NULL. */
+amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n);
+
+/* Debug taps (stream-ordered copy into dst, host or device).  Names and element types:
+ *   "hidden" f32 [n_nodes,d] post-final-norm rows of the last verify; "logits" f32 [n_nodes,V];
+ *   "d_logits" f32 [K,V]; "hp" f32 [K,d] (Eq. 4); "attn_o" f32 [K,d] (Eq. 5);
+ *   "sal_h" f32 [2,d] (Eq. 1: h^1_t, h^2_t of the last row); "tree_tokens", "argmax" i32 [n_nodes];
+ *   "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v": f32 [rows, d] for cache slots 0..rows-1,
+ *   rows = bytes / (4 d), converted from the cache's storage type.
+ * bytes must not exceed the tensor's size. */
+amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t bytes);
+
+/* Synchronises the stream and reports the committed length, the current root token and the
+ * number of rows pending for the adaptation layers.  Any pointer may be NULL.  Also surfaces
+ * device-side errors (AMPH_ERR_TIMEOUT). */
+amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending);
+
+/* Forgets the sequence (caches are logically emptied); weights stay registered. */
+amph_status amph_reset(amph_ctx* ctx);
+
+void amph_destroy(amph_ctx* ctx);
+
+/* Message of the last failure on ctx ("" if none); with ctx == NULL, of the last failed
+ * amph_init / amph_workspace_bytes on this thread.  The string is owned by the library. */
+const char* amph_last_error(const amph_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMPH_H_ */

@@ -1,0 +1,132 @@
+// Internal declarations shared by the kernels and the host scheduler of the Amphista step.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "amph.h"
+
+namespace amph {
+
+typedef unsigned long long u64;
+
+constexpr int kMaxRows = AMPH_MAX_NODES;   // rows one forward call may carry (tree nodes / prefill chunk)
+constexpr int kMaxK = AMPH_MAX_HEADS_K;
+constexpr int kTopkStride = AMPH_TOPK_STRIDE;   // row stride of the top-k id / value tables
+constexpr int kPendMax = kMaxK + 1;        // rows the adaptation layers may have pending
+
+// Per-call row table: where each row of a forward call sits and what it may see.
+// Row r is at rotary position pos[r], writes its key / value to cache slot slot[r] and attends
+// slots [0, base) plus slot base + m for every set bit m of mask[r] (Fig. 5: ancestors only).
+struct RowMeta {
+  int base;
+  int n_rows;
+  int pos[kMaxRows];
+  int slot[kMaxRows];
+  u64 mask[kMaxRows][2];
+};
+
+// Static tree tables built at init (Appendix A.1).
+struct TreeDev {
+  int n_nodes;
+  int parent[kMaxRows];
+  int depth[kMaxRows];
+  int rank[kMaxRows];
+  u64 anc[kMaxRows][2];     // bit m set <=> node m is on the root path of this node (itself included)
+};
+
+// Device-resident decoding state; every kernel reads lengths from here, so a step needs no
+// host round trip.
+struct DevState {
+  int C;                    // committed tokens (cache slots 0..C-1)
+  int root;                 // token chosen for position C
+  int n_pending;            // rows queued for the adaptation layers (positions C-n_pending..C-1)
+  int err;                  // sticky device-side error code (amph_status) or 0
+  int pend_tok[kPendMax + 3];   // token at position (row position + 1) for each pending row
+  // result of the last acceptance
+  int L;                    // accepted tokens (root included)
+  int C_old;                // C before the acceptance
+  int best;                 // deepest accepted node
+  int next_root;
+  int path[kPendMax + 3];
+  int out_tok[kPendMax + 3];
+};
+
+struct KvView {             // one layer's cache: K and V as [n_heads][max_ctx][head_dim]
+  void* k;
+  void* v;
+};
+
+// fp32 partial sums of a projection: value(row, col) = sum_{s < splits} p[s*split_stride + row*ld + col]
+struct PartialView {
+  const float* p;
+  int splits;
+  int ld;                   // row stride in floats (total output features of the launch)
+  size_t split_stride;      // floats between consecutive splits
+};
+
+// ---- launchers (one per kernel family); dtype = AMPH_DTYPE_* of weights / activations / cache
+void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d,
+                  float* x, cudaStream_t st);
+
+// x <- (mode 0: x, mode 1: x + sum P, mode 2: sum P); then, if gain != NULL, RMSNorm of the result
+// into xn (storage dtype) and hid (fp32); with gain == NULL xn / hid receive the plain row.
+// col_off selects the column window of P.
+void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
+                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st);
+
+void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
+                       cudaStream_t st);
+
+// q <- rope(sum P[:, 0:d]); K cache <- rope(sum P[:, d:2d]); V cache <- sum P[:, 2d:3d]
+void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv,
+                     int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st);
+
+struct AttnScratch {
+  float* o;                 // [splits][heads][rows][head_dim]
+  float* ml;                // [splits][heads][rows][2]  (running max, running sum)
+};
+void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out,
+                           int dtype, int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi,
+                           int max_splits, cudaStream_t st);
+
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st);
+
+// cat[r] = [feat[r] ; tok_emb[next[r]]]   (Eq. 1's concatenation)
+void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat,
+                   int dtype, int rows, int d, cudaStream_t st);
+
+struct GemmSeg { const void* w; };
+// P[row][seg*out + o] = sum_k X[row][k] * W_seg[o][k]; plain CUDA-core kernel, one split.
+void launch_gemm_generic(const void* x, int ldx, const GemmSeg* segs, int n_seg, int out, int in,
+                         float* P, int ldp, int rows, int dtype, cudaStream_t st);
+
+// ---- draft-module specific
+void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev, float* last /*[2][d]*/,
+                        void* last_act /*[>=2][d]*/, int dtype, int d, cudaStream_t st);
+// Hp[k] = src_k + silu(sum P[row_k][k*d + :] + b_k) + PE[k]   (Eq. 2-4)
+void launch_mlp_heads(PartialView P, const float* last, const void* const* bias, const void* pe,
+                      float* hp, void* hp_act, int dtype, int K, int n_sal, int d, cudaStream_t st);
+// unmasked attention across the K rows, one block per attention head (Eq. 5)
+void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
+                          cudaStream_t st);
+// per head k: top-c_k of row k of segment k; also stores the row into d_logits[k]
+void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids, float* vals,
+                       float* d_logits, cudaStream_t st);
+void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st);
+
+// ---- control kernels
+void launch_meta_chain(RowMeta* meta, int base, int n_rows, cudaStream_t st);             // prefill chunk
+void launch_meta_pending(RowMeta* meta, const DevState* s, cudaStream_t st);              // adaptation rows
+void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, const int* override_tok,
+                       int* tok, RowMeta* meta, cudaStream_t st);
+void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st);
+void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
+                    int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st);
+void launch_kv_export(KvView kv, int which, int dtype, int rows, int n_heads, int head_dim, int max_ctx,
+                      float* dst, cudaStream_t st);
+void launch_prefill_tail(DevState* s, const int* amax, int last_row, const float* hidden, float* pend_h,
+                         int d, int C, cudaStream_t st);
+
+}  // namespace amph

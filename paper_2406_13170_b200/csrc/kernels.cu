@@ -1,0 +1,813 @@
+// Memory-bound and control kernels of the Amphista step: embedding, fused residual + RMSNorm,
+// rotary embedding + KV write, split-KV tree attention with a bitmask, SwiGLU, the draft
+// module's head kernels (Eq. 2-6), tree construction, greedy acceptance and KV compaction.
+#include <math.h>
+
+#include "amph_internal.cuh"
+
+namespace amph {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+#define AMPH_DISPATCH(dtype, ...)                                    \
+  do {                                                               \
+    if ((dtype) == AMPH_DTYPE_F32) { typedef float T; __VA_ARGS__; } \
+    else { typedef bf16 T; __VA_ARGS__; }                            \
+  } while (0)
+
+__device__ __forceinline__ float sum_partials(const PartialView& P, int row, int col) {
+  const float* p = P.p + (size_t)row * P.ld + col;
+  float acc = p[0];
+  for (int s = 1; s < P.splits; ++s) acc += p[(size_t)s * P.split_stride];   // fixed order: deterministic
+  return acc;
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += red[i];
+  return t;
+}
+
+// --------------------------------------------------------------------------------------------
+// embedding rows
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const T* __restrict__ emb, const int* __restrict__ toks, int vocab, int d,
+                             float* __restrict__ x) {
+  const int r = blockIdx.x;
+  int t = toks[r];
+  t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+  const T* e = emb + (size_t)t * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)r * d + c] = to_f(e[c]);
+}
+
+void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d, float* x,
+                  cudaStream_t st) {
+  AMPH_DISPATCH(dtype, embed_kernel<T><<<rows, 256, 0, st>>>((const T*)tok_emb, toks, vocab, d, x));
+}
+
+// --------------------------------------------------------------------------------------------
+// residual update + RMSNorm (one block per row)
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode,
+                                  const T* __restrict__ gain, T* __restrict__ xn, float* __restrict__ hid,
+                                  float eps, int d) {
+  extern __shared__ float rowbuf[];
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v;
+    if (mode == 0) {
+      v = x[(size_t)r * d + c];
+    } else {
+      v = sum_partials(P, r, col_off + c);
+      if (mode == 1) v += x[(size_t)r * d + c];
+      x[(size_t)r * d + c] = v;
+    }
+    rowbuf[c] = v;
+    ss += v * v;
+  }
+  if (xn == nullptr && hid == nullptr) return;
+  if (gain == nullptr) {                       // plain cast of the updated row
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+      if (xn) xn[(size_t)r * d + c] = from_f<T>(rowbuf[c]);
+      if (hid) hid[(size_t)r * d + c] = rowbuf[c];
+    }
+    return;
+  }
+  const float tot = block_sum(ss, red);
+  const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float n = to_f(gain[c]) * (rowbuf[c] * inv);
+    if (xn) xn[(size_t)r * d + c] = from_f<T>(n);
+    if (hid) hid[(size_t)r * d + c] = n;
+  }
+}
+
+void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
+                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, resid_norm_kernel<T><<<rows, 256, d * sizeof(float), st>>>(
+                           x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d));
+}
+
+// --------------------------------------------------------------------------------------------
+// rotary table for the rows of one call: table[r][i] = (cos, sin)(pos[r] * theta^(-2i/dh))
+// --------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(const RowMeta* __restrict__ meta, const double* __restrict__ inv_freq,
+                                  float2* __restrict__ table, int half) {
+  const int r = blockIdx.x;
+  const double p = (double)meta->pos[r];
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    double s, c;
+    sincos(p * inv_freq[i], &s, &c);
+    table[r * half + i] = make_float2((float)c, (float)s);
+  }
+}
+
+void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
+                       cudaStream_t st) {
+  rope_table_kernel<<<rows, 64, 0, st>>>(meta, inv_freq, table, half);
+}
+
+// --------------------------------------------------------------------------------------------
+// q / k rotation, KV-cache write (one block per row)
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta,
+                                const float2* __restrict__ rope, T* __restrict__ q, T* __restrict__ kc,
+                                T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
+  const int r = blockIdx.x;
+  const int half = dh >> 1, d = n_heads * dh;
+  const bool live = r < meta->n_rows;
+  const int slot = meta->slot[r];
+  const bool store = live && slot >= 0 && slot < max_ctx;
+  for (int idx = threadIdx.x; idx < n_heads * half; idx += blockDim.x) {
+    const int h = idx / half, i = idx - h * half;
+    const float2 cs = rope[r * half + i];
+    const int c0 = h * dh + i, c1 = c0 + half;
+    const float q0 = sum_partials(P, r, c0), q1 = sum_partials(P, r, c1);
+    q[(size_t)r * d + c0] = from_f<T>(q0 * cs.x - q1 * cs.y);
+    q[(size_t)r * d + c1] = from_f<T>(q1 * cs.x + q0 * cs.y);
+    if (store) {
+      const float k0 = sum_partials(P, r, d + c0), k1 = sum_partials(P, r, d + c1);
+      const size_t o = ((size_t)h * max_ctx + slot) * dh + i;
+      kc[o] = from_f<T>(k0 * cs.x - k1 * cs.y);
+      kc[o + half] = from_f<T>(k1 * cs.x + k0 * cs.y);
+      vc[o] = from_f<T>(sum_partials(P, r, 2 * d + c0));
+      vc[o + half] = from_f<T>(sum_partials(P, r, 2 * d + c1));
+    }
+  }
+}
+
+void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv, int dtype,
+                     int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, qkv_rope_kernel<T><<<rows, 256, 0, st>>>(P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
+                                                                n_heads, head_dim, max_ctx));
+}
+
+// --------------------------------------------------------------------------------------------
+// Tree attention, split over the KV axis (flash-decoding form), with the tree as a bitmask.
+// Grid (head, split, row block of 64).  Slots below meta->base are visible to every row;
+// slot base + m is visible to row r iff bit m of mask[r] is set.
+// --------------------------------------------------------------------------------------------
+constexpr int kAttRows = 64;     // query rows per block
+constexpr int kAttTile = 32;     // keys per inner tile
+constexpr int kAttThreads = 256;
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(kAttThreads)
+tree_attn_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
+                 const RowMeta* __restrict__ meta, float* __restrict__ po, float* __restrict__ pml,
+                 int rows_cap, int n_heads, int max_ctx) {
+  constexpr int QS = DH + 4;                       // padded row strides (bank-conflict free float4 reads)
+  constexpr int SEG = DH / 4;                      // output dims owned by one thread
+  extern __shared__ __align__(16) float sm[];
+  float* Qs = sm;                                  // [64][QS]
+  float* Ks = Qs + kAttRows * QS;                  // [32][QS]
+  float* Vs = Ks + kAttTile * QS;                  // [32][DH]
+  float* Ss = Vs + kAttTile * DH;                  // [64][33]
+  const int h = blockIdx.x, split = blockIdx.y, rb = blockIdx.z;
+  const int tid = threadIdx.x;
+  const int r = tid >> 2, qd = tid & 3;
+  const int rg = rb * kAttRows + r;                // global row
+  const int base = meta->base, n_rows = meta->n_rows;
+  const int d = n_heads * DH;
+  const int total = base + n_rows;                 // slots that can be visible
+  int chunk = (total + gridDim.y - 1) / gridDim.y;
+  chunk = (chunk + kAttTile - 1) / kAttTile * kAttTile;
+  const int s_lo = split * chunk;
+  int s_hi = s_lo + chunk;
+  if (s_hi > total) s_hi = total;
+  if (s_hi > max_ctx) s_hi = max_ctx;
+  const bool live = rg < n_rows;
+  u64 m0 = 0, m1 = 0;
+  if (live) { m0 = meta->mask[rg][0]; m1 = meta->mask[rg][1]; }
+  for (int i = tid; i < kAttRows * DH; i += kAttThreads) {
+    const int rr = i / DH, c = i - rr * DH;
+    const int g = rb * kAttRows + rr;
+    Qs[rr * QS + c] = g < rows_cap ? to_f(q[(size_t)g * d + h * DH + c]) : 0.f;
+  }
+  float acc[SEG];
+#pragma unroll
+  for (int i = 0; i < SEG; ++i) acc[i] = 0.f;
+  float mrun = -INFINITY, lrun = 0.f;
+  const float scale = 1.0f / sqrtf((float)DH);
+  const T* kh = kc + (size_t)h * max_ctx * DH;
+  const T* vh = vc + (size_t)h * max_ctx * DH;
+  for (int t0 = s_lo; t0 < s_hi; t0 += kAttTile) {
+    __syncthreads();
+    for (int i = tid; i < kAttTile * DH; i += kAttThreads) {
+      const int j = i / DH, c = i - j * DH;
+      const int s = t0 + j;
+      float kvv = 0.f, vvv = 0.f;
+      if (s < s_hi) { kvv = to_f(kh[(size_t)s * DH + c]); vvv = to_f(vh[(size_t)s * DH + c]); }
+      Ks[j * QS + c] = kvv;
+      Vs[j * DH + c] = vvv;
+    }
+    __syncthreads();
+    float sc[kAttTile / 4];
+    float tmax = -INFINITY;
+#pragma unroll
+    for (int jj = 0; jj < kAttTile / 4; ++jj) {
+      const int j = jj * 4 + qd;
+      const int s = t0 + j;
+      bool vis = live && s < s_hi;
+      if (vis && s >= base) {
+        const int m = s - base;
+        vis = m < 64 ? ((m0 >> m) & 1ull) : ((m1 >> (m - 64)) & 1ull);
+      }
+      float dot = -INFINITY;
+      if (vis) {
+        const float4* qa = reinterpret_cast<const float4*>(Qs + r * QS);
+        const float4* ka = reinterpret_cast<const float4*>(Ks + j * QS);
+        dot = 0.f;
+#pragma unroll 8
+        for (int c = 0; c < DH / 4; ++c) {
+          const float4 a = qa[c], b = ka[c];
+          dot += a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w;
+        }
+        dot *= scale;
+        tmax = fmaxf(tmax, dot);
+      }
+      sc[jj] = dot;
+    }
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+    const float mnew = fmaxf(mrun, tmax);
+    float corr = 1.f, psum = 0.f;
+    if (mnew == -INFINITY) {                       // nothing visible yet for this row
+#pragma unroll
+      for (int jj = 0; jj < kAttTile / 4; ++jj) Ss[r * (kAttTile + 1) + jj * 4 + qd] = 0.f;
+    } else {
+      corr = expf(mrun - mnew);                    // exp(-inf) = 0 on the first visible tile
+#pragma unroll
+      for (int jj = 0; jj < kAttTile / 4; ++jj) {
+        const float p = sc[jj] == -INFINITY ? 0.f : expf(sc[jj] - mnew);
+        Ss[r * (kAttTile + 1) + jj * 4 + qd] = p;
+        psum += p;
+      }
+    }
+    psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+    psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+    lrun = lrun * corr + psum;
+    mrun = mnew;
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < SEG; ++i) acc[i] *= corr;
+    for (int j = 0; j < kAttTile; ++j) {
+      const float p = Ss[r * (kAttTile + 1) + j];
+      if (p != 0.f) {
+        const float4* va = reinterpret_cast<const float4*>(Vs + j * DH + qd * SEG);
+#pragma unroll
+        for (int c = 0; c < SEG / 4; ++c) {
+          const float4 v = va[c];
+          acc[c * 4 + 0] += p * v.x; acc[c * 4 + 1] += p * v.y;
+          acc[c * 4 + 2] += p * v.z; acc[c * 4 + 3] += p * v.w;
+        }
+      }
+    }
+    __syncwarp();
+  }
+  if (rg < rows_cap) {
+    const size_t o = (((size_t)split * n_heads + h) * rows_cap + rg);
+    float4* dst = reinterpret_cast<float4*>(po + o * DH + qd * SEG);
+#pragma unroll
+    for (int c = 0; c < SEG / 4; ++c)
+      dst[c] = make_float4(acc[c * 4], acc[c * 4 + 1], acc[c * 4 + 2], acc[c * 4 + 3]);
+    if (qd == 0) { pml[o * 2] = mrun; pml[o * 2 + 1] = lrun; }
+  }
+}
+
+template <typename T>
+__global__ void attn_combine_kernel(const float* __restrict__ po, const float* __restrict__ pml,
+                                    T* __restrict__ out, int splits, int rows_cap, int n_heads, int dh) {
+  const int r = blockIdx.x, h = blockIdx.y;
+  float M = -INFINITY;
+  for (int s = 0; s < splits; ++s)
+    M = fmaxf(M, pml[(((size_t)s * n_heads + h) * rows_cap + r) * 2]);
+  float den = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const size_t o = ((size_t)s * n_heads + h) * rows_cap + r;
+    const float m = pml[o * 2];
+    if (m != -INFINITY) den += pml[o * 2 + 1] * expf(m - M);
+  }
+  for (int c = threadIdx.x; c < dh; c += blockDim.x) {
+    float num = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const size_t o = ((size_t)s * n_heads + h) * rows_cap + r;
+      const float m = pml[o * 2];
+      if (m != -INFINITY) num += po[o * dh + c] * expf(m - M);
+    }
+    out[(size_t)r * n_heads * dh + h * dh + c] = from_f<T>(den > 0.f ? num / den : 0.f);
+  }
+}
+
+template <typename T, int DH>
+static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out,
+                             int rows, int n_heads, int max_ctx, int splits, cudaStream_t st) {
+  const size_t smem = sizeof(float) * (kAttRows * (DH + 4) + kAttTile * (DH + 4) + kAttTile * DH +
+                                       kAttRows * (kAttTile + 1));
+  cudaFuncSetAttribute(tree_attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  dim3 grid(n_heads, splits, (rows + kAttRows - 1) / kAttRows);
+  tree_attn_kernel<T, DH><<<grid, kAttThreads, smem, st>>>((const T*)q, (const T*)kv.k, (const T*)kv.v, meta,
+                                                          sc.o, sc.ml, rows, n_heads, max_ctx);
+  attn_combine_kernel<T><<<dim3(rows, n_heads), DH < 128 ? 64 : 128, 0, st>>>(sc.o, sc.ml, (T*)out, splits, rows,
+                                                                              n_heads, DH);
+}
+
+void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out, int dtype,
+                           int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi, int max_splits,
+                           cudaStream_t st) {
+  int splits = (ctx_hi + 127) / 128;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  if (head_dim == 64) {
+    AMPH_DISPATCH(dtype, (tree_attention_t<T, 64>(q, kv, meta, sc, out, rows, n_heads, max_ctx, splits, st)));
+  } else {
+    AMPH_DISPATCH(dtype, (tree_attention_t<T, 128>(q, kv, meta, sc, out, rows, n_heads, max_ctx, splits, st)));
+  }
+}
+
+// --------------------------------------------------------------------------------------------
+// SwiGLU on the fused gate / up projection: act = silu(gate) * up
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f) {
+  const size_t n = (size_t)rows * f;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / f), c = (int)(i - (size_t)r * f);
+    const float g = sum_partials(P, r, c), u = sum_partials(P, r, f + c);
+    act[i] = from_f<T>(g / (1.0f + expf(-g)) * u);
+  }
+}
+
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st) {
+  const size_t n = (size_t)rows * f;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  AMPH_DISPATCH(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(P, (T*)act, rows, f));
+}
+
+// --------------------------------------------------------------------------------------------
+// Eq. 1's concatenation [feature ; embedding of the next token]
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void concat_kernel(const float* __restrict__ feat, const T* __restrict__ emb,
+                              const int* __restrict__ next_tok, int vocab, T* __restrict__ cat, int d) {
+  const int r = blockIdx.x;
+  int t = next_tok[r];
+  t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    cat[(size_t)r * 2 * d + c] = from_f<T>(feat[(size_t)r * d + c]);
+    cat[(size_t)r * 2 * d + d + c] = emb[(size_t)t * d + c];
+  }
+}
+
+void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat, int dtype,
+                   int rows, int d, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, concat_kernel<T><<<rows, 256, 0, st>>>(feat, (const T*)tok_emb, next_tok, vocab, (T*)cat, d));
+}
+
+// --------------------------------------------------------------------------------------------
+// Plain projection kernel: one warp per output feature, 128-bit weight loads, fp32 accumulate.
+// Used for fp32 models, for shapes the tensor-core kernel does not cover, and as its A/B check.
+// --------------------------------------------------------------------------------------------
+template <typename T> struct Vec16;
+template <> struct Vec16<float> { static constexpr int N = 4; };
+template <> struct Vec16<bf16> { static constexpr int N = 8; };
+
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float* out);
+template <>
+__device__ __forceinline__ void load16<float>(const float* p, float* out) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <>
+__device__ __forceinline__ void load16<bf16>(const bf16* p, float* out) {
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
+  const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+template <typename T, int R>
+__global__ void __launch_bounds__(256)
+gemm_generic_kernel(const T* __restrict__ X, int ldx, const T* __restrict__ W, int out, int in,
+                    float* __restrict__ P, int ldp, int col_off, int rows) {
+  constexpr int V = Vec16<T>::N;
+  const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (o >= out) return;
+  const T* w = W + (size_t)o * in;
+  for (int r0 = 0; r0 < rows; r0 += R) {
+    float acc[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) acc[i] = 0.f;
+    for (int k = lane * V; k < in; k += 32 * V) {
+      float wv[V];
+      load16<T>(w + k, wv);
+#pragma unroll
+      for (int i = 0; i < R; ++i) {
+        if (r0 + i < rows) {
+          float xv[V];
+          load16<T>(X + (size_t)(r0 + i) * ldx + k, xv);
+#pragma unroll
+          for (int e = 0; e < V; ++e) acc[i] += wv[e] * xv[e];
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      float v = acc[i];
+      for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+      if (lane == 0 && r0 + i < rows) P[(size_t)(r0 + i) * ldp + col_off + o] = v;
+    }
+  }
+}
+
+void launch_gemm_generic(const void* x, int ldx, const GemmSeg* segs, int n_seg, int out, int in, float* P,
+                         int ldp, int rows, int dtype, cudaStream_t st) {
+  const int blocks = (out + 7) / 8;
+  for (int s = 0; s < n_seg; ++s) {
+    AMPH_DISPATCH(dtype, gemm_generic_kernel<T, 8><<<blocks, 256, 0, st>>>(
+                             (const T*)x, ldx, (const T*)segs[s].w, out, in, P, ldp, s * out, rows));
+  }
+}
+
+// --------------------------------------------------------------------------------------------
+// draft module: last-row gather, head MLP epilogue (Eq. 2-4), fused K x K attention (Eq. 5)
+// --------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gather_last_kernel(const float* __restrict__ h1, const float* __restrict__ h2,
+                                   const DevState* __restrict__ s, float* __restrict__ last,
+                                   T* __restrict__ last_act, int d) {
+  int lr = s->n_pending - 1;
+  lr = lr < 0 ? 0 : (lr >= kPendMax ? kPendMax - 1 : lr);
+  const float* src = blockIdx.x == 0 ? h1 : h2;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float v = src[(size_t)lr * d + c];
+    last[(size_t)blockIdx.x * d + c] = v;
+    last_act[(size_t)blockIdx.x * d + c] = from_f<T>(v);
+  }
+}
+
+void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev, float* last, void* last_act,
+                        int dtype, int d, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, gather_last_kernel<T><<<2, 256, 0, st>>>(h1, h2, st_dev, last, (T*)last_act, d));
+}
+
+struct BiasPtrs { const void* b[kMaxK]; };
+
+template <typename T>
+__global__ void mlp_heads_kernel(PartialView P, const float* __restrict__ last, BiasPtrs bias,
+                                 const T* __restrict__ pe, float* __restrict__ hp, T* __restrict__ hp_act,
+                                 int K, int n_sal, int d) {
+  const int k = blockIdx.x;
+  const int row = (k < K / 2 || n_sal == 1) ? 0 : 1;       // Eq. 2: first half of the heads <- stage 1
+  const T* b = (const T*)bias.b[k];
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float pre = sum_partials(P, row, k * d + c) + to_f(b[c]);
+    const float v = last[(size_t)row * d + c] + pre / (1.0f + expf(-pre)) + to_f(pe[(size_t)k * d + c]);
+    hp[(size_t)k * d + c] = v;
+    hp_act[(size_t)k * d + c] = from_f<T>(v);
+  }
+}
+
+void launch_mlp_heads(PartialView P, const float* last, const void* const* bias, const void* pe, float* hp,
+                      void* hp_act, int dtype, int K, int n_sal, int d, cudaStream_t st) {
+  BiasPtrs bp;
+  for (int k = 0; k < kMaxK; ++k) bp.b[k] = k < K ? bias[k] : nullptr;
+  AMPH_DISPATCH(dtype, mlp_heads_kernel<T><<<K, 256, 0, st>>>(P, last, bp, (const T*)pe, hp, (T*)hp_act, K,
+                                                              n_sal, d));
+}
+
+// One block per attention head: the K x K score matrix, softmax and mixing stay in shared memory.
+template <typename T>
+__global__ void aeb_attention_kernel(PartialView P, T* __restrict__ out, int K, int n_heads, int dh) {
+  extern __shared__ float sm[];
+  float* qs = sm;                 // [K][dh]
+  float* ks = qs + K * dh;
+  float* vs = ks + K * dh;
+  float* pr = vs + K * dh;        // [K][K]
+  const int h = blockIdx.x, d = n_heads * dh;
+  for (int i = threadIdx.x; i < K * dh; i += blockDim.x) {
+    const int r = i / dh, c = i - r * dh;
+    qs[i] = sum_partials(P, r, h * dh + c);
+    ks[i] = sum_partials(P, r, d + h * dh + c);
+    vs[i] = sum_partials(P, r, 2 * d + h * dh + c);
+  }
+  __syncthreads();
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int p = w; p < K * K; p += nw) {               // one warp per (i, j) score
+    const int i = p / K, j = p - i * K;
+    float dot = 0.f;
+    for (int c = lane; c < dh; c += 32) dot += qs[i * dh + c] * ks[j * dh + c];
+    for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
+    if (lane == 0) pr[p] = dot / sqrtf((float)dh);
+  }
+  __syncthreads();
+  if (threadIdx.x < K) {                              // bi-directional: every row sees every row
+    const int i = threadIdx.x;
+    float m = -INFINITY;
+    for (int j = 0; j < K; ++j) m = fmaxf(m, pr[i * K + j]);
+    float sum = 0.f;
+    for (int j = 0; j < K; ++j) { const float e = expf(pr[i * K + j] - m); pr[i * K + j] = e; sum += e; }
+    for (int j = 0; j < K; ++j) pr[i * K + j] /= sum;
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < K * dh; idx += blockDim.x) {
+    const int i = idx / dh, c = idx - i * dh;
+    float acc = 0.f;
+    for (int j = 0; j < K; ++j) acc += pr[i * K + j] * vs[j * dh + c];
+    out[(size_t)i * d + h * dh + c] = from_f<T>(acc);
+  }
+}
+
+void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
+                          cudaStream_t st) {
+  const size_t smem = sizeof(float) * (3 * K * head_dim + K * K);
+  AMPH_DISPATCH(dtype, aeb_attention_kernel<T><<<n_heads, 128, smem, st>>>(P, (T*)out_act, K, n_heads, head_dim));
+}
+
+// --------------------------------------------------------------------------------------------
+// selection: top-k per drafting head (Eq. 6), greedy argmax per verified row
+// order: value descending, equal values by ascending id
+// --------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi) {
+  return v > bv || (v == bv && i < bi);
+}
+
+__device__ void block_best(float& v, int& i, float* sv, int* si) {
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+    if (better(ov, oi, v, i)) { v = ov; i = oi; }
+  }
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) { sv[w] = v; si[w] = i; }
+  __syncthreads();
+  v = sv[0]; i = si[0];
+  for (int k = 1; k < nw; ++k)
+    if (better(sv[k], si[k], v, i)) { v = sv[k]; i = si[k]; }
+}
+
+struct TopkCounts { int c[kMaxK]; };
+
+__global__ void topk_heads_kernel(PartialView P, int vocab, TopkCounts ck, int* __restrict__ ids,
+                                  float* __restrict__ vals, float* __restrict__ d_logits) {
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  const int k = blockIdx.x;
+  float* row = d_logits + (size_t)k * vocab;
+  for (int c = threadIdx.x; c < vocab; c += blockDim.x) row[c] = sum_partials(P, k, k * vocab + c);
+  __syncthreads();
+  float pv = INFINITY;
+  int pi = -1;
+  for (int t = 0; t < ck.c[k]; ++t) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
+      const float v = row[c];
+      const bool after_prev = v < pv || (v == pv && c > pi);     // strictly after the previous pick
+      if (after_prev && better(v, c, bv, bi)) { bv = v; bi = c; }
+    }
+    block_best(bv, bi, sv, si);
+    if (threadIdx.x == 0) { ids[k * kTopkStride + t] = bi; vals[k * kTopkStride + t] = bv; }
+    pv = bv; pi = bi;
+    __syncthreads();
+  }
+}
+
+void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids, float* vals, float* d_logits,
+                       cudaStream_t st) {
+  TopkCounts c;
+  for (int k = 0; k < kMaxK; ++k) c.c[k] = k < K ? ck[k] : 0;
+  topk_heads_kernel<<<K, 1024, 0, st>>>(P, vocab, c, ids, vals, d_logits);
+}
+
+__global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ amax,
+                                   float* __restrict__ logits_out) {
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  const int r = blockIdx.x;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
+    const float v = sum_partials(P, r, c);
+    if (logits_out) logits_out[(size_t)r * vocab + c] = v;
+    if (better(v, c, bv, bi)) { bv = v; bi = c; }
+  }
+  block_best(bv, bi, sv, si);
+  if (threadIdx.x == 0) amax[r] = bi;
+}
+
+void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st) {
+  argmax_rows_kernel<<<rows, 1024, 0, st>>>(P, vocab, amax, logits_out);
+}
+
+// --------------------------------------------------------------------------------------------
+// control: row tables, tree tokens, acceptance, compaction
+// --------------------------------------------------------------------------------------------
+__device__ __forceinline__ void chain_mask(int r, u64* m) {       // bits 0..r
+  m[0] = r >= 63 ? ~0ull : ((1ull << (r + 1)) - 1ull);
+  m[1] = r < 64 ? 0ull : (r >= 127 ? ~0ull : ((1ull << (r - 63)) - 1ull));
+}
+
+__global__ void meta_chain_kernel(RowMeta* meta, int base, int n_rows) {
+  const int r = threadIdx.x;
+  if (r == 0) { meta->base = base; meta->n_rows = n_rows; }
+  meta->pos[r] = base + r;
+  meta->slot[r] = base + r;
+  chain_mask(r, meta->mask[r]);
+}
+
+void launch_meta_chain(RowMeta* meta, int base, int n_rows, cudaStream_t st) {
+  meta_chain_kernel<<<1, kMaxRows, 0, st>>>(meta, base, n_rows);
+}
+
+__global__ void meta_pending_kernel(RowMeta* meta, const DevState* s) {
+  const int r = threadIdx.x;
+  int np = s->n_pending;
+  np = np < 0 ? 0 : (np > kPendMax ? kPendMax : np);
+  const int base = s->C - np;
+  if (r == 0) { meta->base = base; meta->n_rows = np; }
+  meta->pos[r] = base + r;
+  meta->slot[r] = base + r;
+  chain_mask(r, meta->mask[r]);
+}
+
+void launch_meta_pending(RowMeta* meta, const DevState* s, cudaStream_t st) {
+  meta_pending_kernel<<<1, kMaxRows, 0, st>>>(meta, s);
+}
+
+// tok[0] = root; tok[n] = head depth[n]'s candidate of rank rank[n] (Appendix A.1); optional overrides;
+// row table of the verification pass: position C + depth, slot C + n, mask = ancestors (Fig. 5).
+__global__ void tree_build_kernel(const TreeDev* __restrict__ tree, DevState* s, const int* __restrict__ topk_ids,
+                                  const int* __restrict__ override_tok, int* __restrict__ tok, RowMeta* meta) {
+  const int n = threadIdx.x;
+  const int N = tree->n_nodes;
+  const int C = s->C;
+  if (n == 0) { meta->base = C; meta->n_rows = N; }
+  if (n < N) {
+    if (n == 0) {
+      tok[0] = s->root;
+    } else {
+      if (topk_ids) tok[n] = topk_ids[(tree->depth[n] - 1) * kTopkStride + tree->rank[n]];
+      if (override_tok && override_tok[n] >= 0) tok[n] = override_tok[n];
+    }
+    meta->pos[n] = C + tree->depth[n];
+    meta->slot[n] = C + n;
+    meta->mask[n][0] = tree->anc[n][0];
+    meta->mask[n][1] = tree->anc[n][1];
+  } else {
+    meta->pos[n] = C;
+    meta->slot[n] = -1;
+    meta->mask[n][0] = meta->mask[n][1] = 0ull;
+  }
+}
+
+void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, const int* override_tok, int* tok,
+                       RowMeta* meta, cudaStream_t st) {
+  tree_build_kernel<<<1, kMaxRows, 0, st>>>(tree, s, topk_ids, override_tok, tok, meta);
+}
+
+// Greedy acceptance: node n matches if its token equals the target's choice at its parent; it is
+// accepted if every node on its root path matches; the deepest accepted node wins (lowest index
+// among equals).  One block; the match set is a 128-bit mask tested against the ancestor masks.
+__global__ void accept_kernel(const TreeDev* __restrict__ tree, DevState* s, const int* __restrict__ tok,
+                              const int* __restrict__ amax) {
+  __shared__ u64 match[2];
+  __shared__ int best_key;
+  const int n = threadIdx.x;
+  const int N = tree->n_nodes;
+  if (n < 2) match[n] = 0ull;
+  if (n == 0) best_key = 0;
+  __syncthreads();
+  if (n < N) {
+    const bool m = n == 0 || tok[n] == amax[tree->parent[n]];
+    if (m) atomicOr(&match[n >> 6], 1ull << (n & 63));
+  }
+  __syncthreads();
+  if (n < N) {
+    const bool ok = ((tree->anc[n][0] & ~match[0]) | (tree->anc[n][1] & ~match[1])) == 0ull;
+    if (ok) atomicMax(&best_key, tree->depth[n] * 256 + (255 - n));
+  }
+  __syncthreads();
+  if (n == 0) {
+    const int best = 255 - (best_key & 255);
+    const int C = s->C;
+    u64 a0 = tree->anc[best][0], a1 = tree->anc[best][1];
+    int L = 0;
+    while (a0 && L < kPendMax) { s->path[L++] = __ffsll((long long)a0) - 1; a0 &= a0 - 1; }
+    while (a1 && L < kPendMax) { s->path[L++] = 64 + __ffsll((long long)a1) - 1; a1 &= a1 - 1; }
+    const int nr = amax[best];
+    for (int j = 0; j < L; ++j) {
+      s->out_tok[j] = tok[s->path[j]];
+      s->pend_tok[j] = j + 1 < L ? tok[s->path[j + 1]] : nr;
+    }
+    for (int j = L; j < kPendMax; ++j) { s->path[j] = -1; s->out_tok[j] = -1; }
+    s->L = L;
+    s->C_old = C;
+    s->best = best;
+    s->next_root = nr;
+    s->C = C + L;
+    s->root = nr;
+    s->n_pending = L;
+  }
+}
+
+void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st) {
+  accept_kernel<<<1, kMaxRows, 0, st>>>(tree, s, tok, amax);
+}
+
+// Block l < n_layers moves layer l's accepted key / value rows: slot C_old + j <- C_old + path[j].
+// path is strictly increasing with path[j] >= j, so no source is overwritten before it is read and
+// the moves are independent.  The extra last block queues the accepted hidden rows for the next draft.
+template <typename T>
+__global__ void compact_kernel(const DevState* __restrict__ s, const KvView* __restrict__ kv, int n_layers,
+                               int n_heads, int dh, int max_ctx, const float* __restrict__ hidden,
+                               float* __restrict__ pend_h, int d) {
+  const int L = s->L, C0 = s->C_old;
+  if ((int)blockIdx.x == n_layers) {
+    for (int j = 0; j < L; ++j)
+      for (int c = threadIdx.x; c < d; c += blockDim.x) pend_h[(size_t)j * d + c] = hidden[(size_t)s->path[j] * d + c];
+    return;
+  }
+  T* kc = (T*)kv[blockIdx.x].k;
+  T* vc = (T*)kv[blockIdx.x].v;
+  for (int j = 1; j < L; ++j) {
+    const int src = C0 + s->path[j], dst = C0 + j;
+    if (src == dst || src >= max_ctx) continue;
+    for (int i = threadIdx.x; i < n_heads * dh; i += blockDim.x) {
+      const int h = i / dh, c = i - h * dh;
+      const size_t so = ((size_t)h * max_ctx + src) * dh + c, dd = ((size_t)h * max_ctx + dst) * dh + c;
+      kc[dd] = kc[so];
+      vc[dd] = vc[so];
+    }
+  }
+}
+
+void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
+                    int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, compact_kernel<T><<<n_layers + 1, 256, 0, st>>>(s, kv_layers, n_layers, n_heads, head_dim,
+                                                                       max_ctx, hidden, pend_h, d));
+}
+
+template <typename T>
+__global__ void kv_export_kernel(const T* __restrict__ c, int n_heads, int dh, int max_ctx, float* __restrict__ dst) {
+  const int slot = blockIdx.x;
+  for (int i = threadIdx.x; i < n_heads * dh; i += blockDim.x) {
+    const int h = i / dh, e = i - h * dh;
+    dst[(size_t)slot * n_heads * dh + i] = to_f(c[((size_t)h * max_ctx + slot) * dh + e]);
+  }
+}
+
+void launch_kv_export(KvView kv, int which, int dtype, int rows, int n_heads, int head_dim, int max_ctx,
+                      float* dst, cudaStream_t st) {
+  if (rows <= 0) return;
+  AMPH_DISPATCH(dtype, kv_export_kernel<T><<<rows, 256, 0, st>>>((const T*)(which ? kv.v : kv.k), n_heads,
+                                                                 head_dim, max_ctx, dst));
+}
+
+// End of prefill: root = greedy choice after the last prompt token; the last prompt row stays
+// pending so that the first draft runs the adaptation layers on it (Eq. 1).
+__global__ void prefill_tail_kernel(DevState* s, const int* __restrict__ amax, int last_row,
+                                    const float* __restrict__ hidden, float* __restrict__ pend_h, int d, int C) {
+  for (int c = threadIdx.x; c < d; c += blockDim.x) pend_h[c] = hidden[(size_t)last_row * d + c];
+  if (threadIdx.x == 0) {
+    const int root = amax[last_row];
+    s->C = C;
+    s->root = root;
+    s->n_pending = 1;
+    s->pend_tok[0] = root;
+    s->L = 0;
+    s->C_old = C;
+    s->best = 0;
+    s->next_root = root;
+  }
+}
+
+void launch_prefill_tail(DevState* s, const int* amax, int last_row, const float* hidden, float* pend_h, int d,
+                         int C, cudaStream_t st) {
+  prefill_tail_kernel<<<1, 256, 0, st>>>(s, amax, last_row, hidden, pend_h, d, C);
+}
+
+}  // namespace amph
