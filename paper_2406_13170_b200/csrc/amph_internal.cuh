@@ -43,14 +43,14 @@ struct DevState {
   int root;                 // token chosen for position C
   int n_pending;            // rows queued for the adaptation layers (positions C-n_pending..C-1)
   int err;                  // sticky device-side error code (amph_status) or 0
-  int pend_tok[kPendMax + 3];   // token at position (row position + 1) for each pending row
+  int pend_tok[16];         // token at position (row position + 1) for each pending row
   // result of the last acceptance
   int L;                    // accepted tokens (root included)
   int C_old;                // C before the acceptance
   int best;                 // deepest accepted node
   int next_root;
-  int path[kPendMax + 3];
-  int out_tok[kPendMax + 3];
+  int path[16];
+  int out_tok[16];
 };
 
 struct KvView {             // one layer's cache: K and V as [n_heads][max_ctx][head_dim]
@@ -107,7 +107,7 @@ void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev
                         void* last_act /*[>=2][d]*/, int dtype, int d, cudaStream_t st);
 // Hp[k] = src_k + silu(sum P[row_k][k*d + :] + b_k) + PE[k]   (Eq. 2-4)
 void launch_mlp_heads(PartialView P, const float* last, const void* const* bias, const void* pe,
-                      float* hp, void* hp_act, int dtype, int K, int n_sal, int d, cudaStream_t st);
+                      float* hp, float* ao, void* ao_act, int dtype, int K, int n_sal, int d, cudaStream_t st);
 // unmasked attention across the K rows, one block per attention head (Eq. 5)
 void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
                           cudaStream_t st);
@@ -124,7 +124,7 @@ void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, co
 void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st);
 void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
                     int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st);
-void launch_kv_export(KvView kv, int which, int dtype, int rows, int n_heads, int head_dim, int max_ctx,
+void launch_kv_export(KvView kv, int which, int dtype, int row0, int rows, int n_heads, int head_dim, int max_ctx,
                       float* dst, cudaStream_t st);
 void launch_prefill_tail(DevState* s, const int* amax, int last_row, const float* hidden, float* pend_h,
                          int d, int C, cudaStream_t st);

@@ -477,8 +477,8 @@ struct BiasPtrs { const void* b[kMaxK]; };
 
 template <typename T>
 __global__ void mlp_heads_kernel(PartialView P, const float* __restrict__ last, BiasPtrs bias,
-                                 const T* __restrict__ pe, float* __restrict__ hp, T* __restrict__ hp_act,
-                                 int K, int n_sal, int d) {
+                                 const T* __restrict__ pe, float* __restrict__ hp, float* __restrict__ ao,
+                                 T* __restrict__ ao_act, int K, int n_sal, int d) {
   const int k = blockIdx.x;
   const int row = (k < K / 2 || n_sal == 1) ? 0 : 1;       // Eq. 2: first half of the heads <- stage 1
   const T* b = (const T*)bias.b[k];
@@ -486,16 +486,17 @@ __global__ void mlp_heads_kernel(PartialView P, const float* __restrict__ last, 
     const float pre = sum_partials(P, row, k * d + c) + to_f(b[c]);
     const float v = last[(size_t)row * d + c] + pre / (1.0f + expf(-pre)) + to_f(pe[(size_t)k * d + c]);
     hp[(size_t)k * d + c] = v;
-    hp_act[(size_t)k * d + c] = from_f<T>(v);
+    ao[(size_t)k * d + c] = v;                // the attention block updates this copy in place
+    ao_act[(size_t)k * d + c] = from_f<T>(v);
   }
 }
 
 void launch_mlp_heads(PartialView P, const float* last, const void* const* bias, const void* pe, float* hp,
-                      void* hp_act, int dtype, int K, int n_sal, int d, cudaStream_t st) {
+                      float* ao, void* ao_act, int dtype, int K, int n_sal, int d, cudaStream_t st) {
   BiasPtrs bp;
   for (int k = 0; k < kMaxK; ++k) bp.b[k] = k < K ? bias[k] : nullptr;
-  AMPH_DISPATCH(dtype, mlp_heads_kernel<T><<<K, 256, 0, st>>>(P, last, bp, (const T*)pe, hp, (T*)hp_act, K,
-                                                              n_sal, d));
+  AMPH_DISPATCH(dtype, mlp_heads_kernel<T><<<K, 256, 0, st>>>(P, last, bp, (const T*)pe, hp, ao, (T*)ao_act,
+                                                              K, n_sal, d));
 }
 
 // One block per attention head: the K x K score matrix, softmax and mixing stay in shared memory.
@@ -772,18 +773,19 @@ void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, in
 }
 
 template <typename T>
-__global__ void kv_export_kernel(const T* __restrict__ c, int n_heads, int dh, int max_ctx, float* __restrict__ dst) {
-  const int slot = blockIdx.x;
+__global__ void kv_export_kernel(const T* __restrict__ c, int row0, int n_heads, int dh, int max_ctx,
+                                 float* __restrict__ dst) {
+  const int slot = row0 + blockIdx.x;
   for (int i = threadIdx.x; i < n_heads * dh; i += blockDim.x) {
     const int h = i / dh, e = i - h * dh;
-    dst[(size_t)slot * n_heads * dh + i] = to_f(c[((size_t)h * max_ctx + slot) * dh + e]);
+    dst[(size_t)blockIdx.x * n_heads * dh + i] = to_f(c[((size_t)h * max_ctx + slot) * dh + e]);
   }
 }
 
-void launch_kv_export(KvView kv, int which, int dtype, int rows, int n_heads, int head_dim, int max_ctx,
+void launch_kv_export(KvView kv, int which, int dtype, int row0, int rows, int n_heads, int head_dim, int max_ctx,
                       float* dst, cudaStream_t st) {
   if (rows <= 0) return;
-  AMPH_DISPATCH(dtype, kv_export_kernel<T><<<rows, 256, 0, st>>>((const T*)(which ? kv.v : kv.k), n_heads,
+  AMPH_DISPATCH(dtype, kv_export_kernel<T><<<rows, 256, 0, st>>>((const T*)(which ? kv.v : kv.k), row0, n_heads,
                                                                  head_dim, max_ctx, dst));
 }
 
