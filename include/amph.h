@@ -172,6 +172,11 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n);
  * bytes must not exceed the tensor's size. */
 amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t bytes);
 
+/* Test hook: overwrites "tree_tokens" or "argmax" (i32 [n_nodes], host or device source) with a
+ * stream-ordered copy, e.g. to run amph_accept on a chosen verification outcome.  Allowed after
+ * amph_verify_tree only. */
+amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes);
+
 /* Synchronises the stream and reports the committed length, the current root token and the
  * number of rows pending for the adaptation layers.  Any pointer may be NULL.  Also surfaces
  * device-side errors (AMPH_ERR_TIMEOUT). */

@@ -1,0 +1,739 @@
+// Host side of the Amphista step library: argument validation, workspace layout, weight
+// registry and the kernel schedule of prefill / draft / verify / accept (declared in amph.h).
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "amph_internal.cuh"
+#include "gemm_tc.cuh"
+
+using namespace amph;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+struct LayerW {
+  const void *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *w_gate, *w_up, *w_down;
+};
+
+struct TensorRec {
+  const void* ptr;
+  int ndim;
+  int64_t shape[2];
+};
+
+// Offsets of every buffer inside the caller's workspace region.
+struct Layout {
+  size_t total = 0;
+  size_t take(size_t bytes) {
+    const size_t off = total;
+    total += (bytes + 255) / 256 * 256;
+    return off;
+  }
+  size_t state, tree, meta_v, meta_s, kv_tab, inv_freq, rope_v, rope_s;
+  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals;
+  size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
+  size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
+  size_t partial, att_o, att_ml, logits, d_logits;
+  size_t partial_floats;
+  int attn_splits;
+};
+
+enum Phase { PH_CREATED = 0, PH_READY, PH_DRAFTED, PH_VERIFIED };
+
+}  // namespace
+
+struct amph_ctx {
+  amph_config cfg;
+  TreeDev tree_host;
+  cudaStream_t stream;
+  int dtype;
+  size_t esz;
+  int Mcap;                 // rows carried by a verification / prefill-chunk pass
+  int rows_small;           // rows carried by the draft module's passes
+  Layout lay;
+  char* ws;
+  char* kv;
+  std::vector<KvView> kv_target;
+  KvView kv_sal[2];
+  std::unordered_map<std::string, TensorRec> tensors;
+  bool resolved;
+  const void *tok_emb, *final_norm, *lm_head, *fc[2], *pe;
+  std::vector<LayerW> layers;
+  LayerW sal[2];
+  const void* mlp_w[kMaxK];
+  const void* mlp_b[kMaxK];
+  const void* aeb_w[2][4];
+  const void* draft_lm[kMaxK];
+  Phase phase;
+  int ctx_hi;               // host-side upper bound of the committed length
+  std::string err;
+  TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+amph_status fail(amph_ctx* ctx, amph_status code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->err = buf;
+  g_last_error = buf;
+  return code;
+}
+
+amph_status cuda_check(amph_ctx* ctx, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return AMPH_OK;
+  return fail(ctx, AMPH_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
+  if (!c || !t) return fail(nullptr, AMPH_ERR_INVALID_ARG, "config and tree must not be NULL");
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ffn < 8 || c->vocab < 2)
+    return fail(nullptr, AMPH_ERR_SHAPE, "non-positive model dimension");
+  if (c->n_heads * c->head_dim != c->d_model)
+    return fail(nullptr, AMPH_ERR_SHAPE, "n_heads * head_dim (%d) != d_model (%d)", c->n_heads * c->head_dim, c->d_model);
+  if (c->head_dim != 64 && c->head_dim != 128)
+    return fail(nullptr, AMPH_ERR_SHAPE, "head_dim must be 64 or 128 (got %d)", c->head_dim);
+  if (c->d_model % 8 || c->d_ffn % 8) return fail(nullptr, AMPH_ERR_SHAPE, "d_model and d_ffn must be multiples of 8");
+  if (c->d_model > 12288) return fail(nullptr, AMPH_ERR_SHAPE, "d_model > 12288 is not supported");
+  if (c->weight_dtype != AMPH_DTYPE_F32 && c->weight_dtype != AMPH_DTYPE_BF16)
+    return fail(nullptr, AMPH_ERR_SHAPE, "unknown weight_dtype %d", c->weight_dtype);
+  if (c->kv_dtype != c->weight_dtype) return fail(nullptr, AMPH_ERR_SHAPE, "kv_dtype must equal weight_dtype");
+  if (c->max_batch != 1) return fail(nullptr, AMPH_ERR_SHAPE, "max_batch must be 1");
+  if (c->K < 1 || c->K > kMaxK) return fail(nullptr, AMPH_ERR_SHAPE, "K must be in 1..%d", kMaxK);
+  if (c->n_sal != 1 && c->n_sal != 2) return fail(nullptr, AMPH_ERR_SHAPE, "n_sal must be 1 or 2");
+  if (c->aeb_layers != 1 && c->aeb_layers != 2) return fail(nullptr, AMPH_ERR_SHAPE, "aeb_layers must be 1 or 2");
+  for (int k = 0; k < c->K; ++k)
+    if (c->topk[k] < 1 || c->topk[k] > kTopkStride || c->topk[k] > c->vocab)
+      return fail(nullptr, AMPH_ERR_SHAPE, "topk[%d] = %d out of range 1..%d", k, c->topk[k], kTopkStride);
+  if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 1.f)) return fail(nullptr, AMPH_ERR_SHAPE, "bad rms_eps / rope_theta");
+  if (t->n_nodes < 1 || t->n_nodes > kMaxRows) return fail(nullptr, AMPH_ERR_SHAPE, "n_nodes must be in 1..%d", kMaxRows);
+  if (!t->parent || !t->depth || !t->rank) return fail(nullptr, AMPH_ERR_INVALID_ARG, "tree arrays must not be NULL");
+  if (c->max_ctx < t->n_nodes + 1) return fail(nullptr, AMPH_ERR_SHAPE, "max_ctx must exceed n_nodes");
+  TreeDev td;
+  memset(&td, 0, sizeof td);
+  td.n_nodes = t->n_nodes;
+  for (int n = 0; n < t->n_nodes; ++n) {
+    const int p = t->parent[n], dep = t->depth[n];
+    if (n == 0) {
+      if (p != -1 || dep != 0) return fail(nullptr, AMPH_ERR_SHAPE, "node 0 must be the root (parent -1, depth 0)");
+      td.anc[0][0] = 1ull;
+    } else {
+      if (p < 0 || p >= n) return fail(nullptr, AMPH_ERR_SHAPE, "parent[%d] = %d must be in 0..%d", n, p, n - 1);
+      if (dep != td.depth[p] + 1) return fail(nullptr, AMPH_ERR_SHAPE, "depth[%d] must be depth[parent] + 1", n);
+      if (dep > c->K) return fail(nullptr, AMPH_ERR_SHAPE, "depth[%d] = %d exceeds K = %d", n, dep, c->K);
+      if (t->rank[n] >= c->topk[dep - 1])
+        return fail(nullptr, AMPH_ERR_SHAPE, "rank[%d] = %d needs topk[%d] > %d", n, t->rank[n], dep - 1, t->rank[n]);
+      td.anc[n][0] = td.anc[p][0];
+      td.anc[n][1] = td.anc[p][1];
+      td.anc[n][n >> 6] |= 1ull << (n & 63);
+    }
+    td.parent[n] = p;
+    td.depth[n] = dep;
+    td.rank[n] = t->rank[n];
+  }
+  if (out) *out = td;
+  return AMPH_OK;
+}
+
+void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, size_t* kv_bytes) {
+  const int Mcap = round_up(n_nodes < 16 ? 16 : n_nodes, 16);
+  const size_t esz = c.weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
+  const size_t d = c.d_model, F = c.d_ffn, V = c.vocab, half = c.head_dim / 2;
+  Layout l;
+  l.state = l.take(sizeof(DevState));
+  l.tree = l.take(sizeof(TreeDev));
+  l.meta_v = l.take(sizeof(RowMeta));
+  l.meta_s = l.take(sizeof(RowMeta));
+  l.kv_tab = l.take(sizeof(KvView) * c.n_layers);
+  l.inv_freq = l.take(sizeof(double) * half);
+  l.rope_v = l.take(sizeof(float2) * Mcap * half);
+  l.rope_s = l.take(sizeof(float2) * Mcap * half);
+  l.tok = l.take(sizeof(int) * kMaxRows);
+  l.amax = l.take(sizeof(int) * kMaxRows);
+  l.override_tok = l.take(sizeof(int) * kMaxRows);
+  l.next_tok = l.take(sizeof(int) * kMaxRows);
+  l.topk_ids = l.take(sizeof(int) * kMaxK * kTopkStride);
+  l.topk_vals = l.take(sizeof(float) * kMaxK * kTopkStride);
+  l.x = l.take(4 * Mcap * d);
+  l.hidden = l.take(4 * Mcap * d);
+  l.h1 = l.take(4 * Mcap * d);
+  l.h2 = l.take(4 * Mcap * d);
+  l.pend_h = l.take(4 * 16 * d);
+  l.last = l.take(4 * 2 * d);
+  l.hp = l.take(4 * kMaxK * d);
+  l.attn_o = l.take(4 * 16 * d);
+  l.xn = l.take(esz * Mcap * d);
+  l.q = l.take(esz * Mcap * d);
+  l.att = l.take(esz * Mcap * d);
+  l.act = l.take(esz * Mcap * F);
+  l.cat = l.take(esz * Mcap * 2 * d);
+  l.last_act = l.take(esz * 16 * d);
+  l.ao_act = l.take(esz * 16 * d);
+  l.aeb_act = l.take(esz * 16 * d);
+  size_t big = 3 * d > 2 * F ? 3 * d : 2 * F;
+  size_t pf = 4 * (size_t)Mcap * big;                       // room for 4 K-splits of the widest projection
+  if (2 * (size_t)Mcap * V > pf) pf = 2 * (size_t)Mcap * V;
+  if ((size_t)16 * c.K * V > pf) pf = (size_t)16 * c.K * V;
+  l.partial_floats = pf;
+  l.partial = l.take(4 * pf);
+  int splits = (296 + c.n_heads - 1) / c.n_heads;
+  if (splits > 16) splits = 16;
+  l.attn_splits = splits;
+  l.att_o = l.take(4 * (size_t)splits * c.n_heads * Mcap * c.head_dim);
+  l.att_ml = l.take(4 * (size_t)splits * c.n_heads * Mcap * 2);
+  l.logits = l.take(4 * (size_t)Mcap * V);
+  l.d_logits = l.take(4 * (size_t)kMaxK * V);
+  *L = l;
+  *Mcap_out = Mcap;
+  const size_t per_layer = 2 * (size_t)c.n_heads * c.max_ctx * c.head_dim * esz;
+  *kv_bytes = per_layer * (c.n_layers + c.n_sal);
+}
+
+// ---- weights ------------------------------------------------------------------------------
+const void* find(amph_ctx* ctx, const std::string& name, int64_t s0, int64_t s1, bool* ok) {
+  auto it = ctx->tensors.find(name);
+  if (it == ctx->tensors.end()) {
+    if (*ok) fail(ctx, AMPH_ERR_MISSING_WEIGHT, "weight '%s' was never loaded", name.c_str());
+    *ok = false;
+    return nullptr;
+  }
+  const TensorRec& t = it->second;
+  const bool shape_ok = s1 == 0 ? (t.ndim == 1 && t.shape[0] == s0) : (t.ndim == 2 && t.shape[0] == s0 && t.shape[1] == s1);
+  if (!shape_ok) {
+    if (*ok) fail(ctx, AMPH_ERR_MISSING_WEIGHT, "weight '%s' has the wrong shape", name.c_str());
+    *ok = false;
+    return nullptr;
+  }
+  return t.ptr;
+}
+
+bool resolve_layer(amph_ctx* ctx, const std::string& pre, LayerW* w, bool* ok) {
+  const int64_t d = ctx->cfg.d_model, F = ctx->cfg.d_ffn;
+  w->attn_norm = find(ctx, pre + "attn_norm", d, 0, ok);
+  w->wq = find(ctx, pre + "wq", d, d, ok);
+  w->wk = find(ctx, pre + "wk", d, d, ok);
+  w->wv = find(ctx, pre + "wv", d, d, ok);
+  w->wo = find(ctx, pre + "wo", d, d, ok);
+  w->ffn_norm = find(ctx, pre + "ffn_norm", d, 0, ok);
+  w->w_gate = find(ctx, pre + "w_gate", F, d, ok);
+  w->w_up = find(ctx, pre + "w_up", F, d, ok);
+  w->w_down = find(ctx, pre + "w_down", d, F, ok);
+  return *ok;
+}
+
+amph_status resolve(amph_ctx* ctx) {
+  if (ctx->resolved) return AMPH_OK;
+  const amph_config& c = ctx->cfg;
+  const int64_t d = c.d_model, V = c.vocab;
+  bool ok = true;
+  ctx->tok_emb = find(ctx, "tok_emb", V, d, &ok);
+  ctx->final_norm = find(ctx, "final_norm", d, 0, &ok);
+  ctx->lm_head = find(ctx, "lm_head", V, d, &ok);
+  ctx->layers.resize(c.n_layers);
+  for (int i = 0; i < c.n_layers; ++i) resolve_layer(ctx, "layers." + std::to_string(i) + ".", &ctx->layers[i], &ok);
+  for (int s = 0; s < c.n_sal; ++s) {
+    ctx->fc[s] = find(ctx, "draft.fc" + std::to_string(s + 1), d, 2 * d, &ok);
+    resolve_layer(ctx, "draft.sal" + std::to_string(s + 1) + ".", &ctx->sal[s], &ok);
+  }
+  for (int k = 0; k < c.K; ++k) {
+    ctx->mlp_w[k] = find(ctx, "draft.mlp." + std::to_string(k) + ".w", d, d, &ok);
+    ctx->mlp_b[k] = find(ctx, "draft.mlp." + std::to_string(k) + ".b", d, 0, &ok);
+    ctx->draft_lm[k] = find(ctx, "draft.lm_head." + std::to_string(k), V, d, &ok);
+  }
+  ctx->pe = find(ctx, "draft.pe", c.K, d, &ok);
+  static const char* names[4] = {"wq", "wk", "wv", "wo"};
+  for (int l = 0; l < c.aeb_layers; ++l)
+    for (int j = 0; j < 4; ++j)
+      ctx->aeb_w[l][j] = find(ctx, "draft.aeb." + std::to_string(l) + "." + names[j], d, d, &ok);
+  if (!ok) return AMPH_ERR_MISSING_WEIGHT;
+  ctx->resolved = true;
+  return AMPH_OK;
+}
+
+// ---- projections --------------------------------------------------------------------------
+// Y = X W^T for up to four weight matrices that share X; the result is left as fp32 partial sums.
+enum XBuf { XB_XN = 0, XB_ATT, XB_ACT, XB_CAT, XB_LAST, XB_AO, XB_AEB, XB_COUNT };
+
+void* xbuf_ptr(amph_ctx* ctx, int xb) {
+  const Layout& l = ctx->lay;
+  const size_t off[XB_COUNT] = {l.xn, l.att, l.act, l.cat, l.last_act, l.ao_act, l.aeb_act};
+  return ctx->ws + off[xb];
+}
+
+PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
+  float* P = ctx->at<float>(ctx->lay.partial);
+  PartialView pv;
+  if (ctx->tc) {
+    int splits = 0;
+    size_t stride = 0;
+    if (tc_gemm_launch(ctx->tc, xb, w, n_seg, out, in, rows, P, ctx->lay.partial_floats, &splits, &stride,
+                       ctx->stream)) {
+      pv.p = P;
+      pv.splits = splits;
+      pv.ld = n_seg * out;
+      pv.split_stride = stride;
+      return pv;
+    }
+  }
+  GemmSeg segs[kMaxK];
+  for (int s = 0; s < n_seg; ++s) segs[s].w = w[s];
+  launch_gemm_generic(xbuf_ptr(ctx, xb), in, segs, n_seg, out, in, P, n_seg * out, rows, ctx->dtype, ctx->stream);
+  pv.p = P;
+  pv.splits = 1;
+  pv.ld = n_seg * out;
+  pv.split_stride = 0;
+  return pv;
+}
+
+// One decoder layer over the rows described by `meta`.  On entry xn holds RMSNorm(x) * attn_norm;
+// on exit x is updated and, if next_gain is given, xn (and hid) hold RMSNorm(x) * next_gain.
+void layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
+                   int rows, int ctx_hi, const void* next_gain, float* hid) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  const void* qkv[3] = {w.wq, w.wk, w.wv};
+  PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
+  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st);
+  AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
+  launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
+                        c.max_ctx, ctx_hi, l.attn_splits, st);
+  const void* wo[1] = {w.wo};
+  P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
+  launch_resid_norm(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows, c.d_model, st);
+  const void* gu[2] = {w.w_gate, w.w_up};
+  P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
+  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st);
+  const void* wd[1] = {w.w_down};
+  P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
+  launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, next_gain ? ctx->ws + l.xn : nullptr, hid, c.rms_eps, rows,
+                    c.d_model, st);
+}
+
+// Target forward of the rows in `tok` under meta_v; leaves post-final-norm rows in hidden and xn.
+void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  const RowMeta* meta = ctx->at<RowMeta>(l.meta_v);
+  float2* rope = ctx->at<float2>(l.rope_v);
+  float* x = ctx->at<float>(l.x);
+  launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
+  launch_embed(ctx->tok_emb, ctx->dtype, ctx->at<int>(l.tok), c.vocab, rows, c.d_model, x, st);
+  PartialView none = {nullptr, 0, 0, 0};
+  launch_resid_norm(x, none, 0, 0, ctx->layers[0].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
+                    c.d_model, st);
+  for (int i = 0; i < c.n_layers; ++i) {
+    const bool last = i + 1 == c.n_layers;
+    layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
+                  last ? ctx->final_norm : ctx->layers[i + 1].attn_norm, last ? ctx->at<float>(l.hidden) : nullptr);
+  }
+}
+
+void target_head(amph_ctx* ctx, int rows) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  const void* w[1] = {ctx->lm_head};
+  PartialView P = project(ctx, XB_XN, w, 1, c.vocab, c.d_model, rows);
+  launch_argmax_rows(P, c.vocab, rows, ctx->at<int>(l.amax), ctx->at<float>(l.logits), ctx->stream);
+}
+
+// Eq. 1: both adaptation stages over the rows (feat, next_tok) described by meta_s.
+void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, int ctx_hi) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  const RowMeta* meta = ctx->at<RowMeta>(l.meta_s);
+  float2* rope = ctx->at<float2>(l.rope_s);
+  launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
+  const float* in_feat = feat;
+  for (int s = 0; s < c.n_sal; ++s) {
+    float* hbuf = ctx->at<float>(s == 0 ? l.h1 : l.h2);
+    launch_concat(in_feat, ctx->tok_emb, next_tok, c.vocab, ctx->ws + l.cat, ctx->dtype, rows, c.d_model, st);
+    const void* w[1] = {ctx->fc[s]};
+    PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, 2 * c.d_model, rows);
+    launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
+                      c.d_model, st);
+    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr);
+    in_feat = hbuf;
+  }
+}
+
+amph_status copy_out(amph_ctx* ctx, void* dst, const void* src, size_t bytes) {
+  if (!dst) return AMPH_OK;
+  return cuda_check(ctx, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, ctx->stream), "copy of a result");
+}
+
+amph_status finish(amph_ctx* ctx, const char* what) { return cuda_check(ctx, cudaGetLastError(), what); }
+
+amph_status refresh_ctx_hi(amph_ctx* ctx) {
+  DevState s;
+  cudaError_t e = cudaMemcpyAsync(&s, ctx->at<DevState>(ctx->lay.state), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_check(ctx, e, "state read-back");
+  ctx->ctx_hi = s.C;
+  if (s.err) return fail(ctx, s.err, "a device-side wait gave up (code %d)", s.err);
+  return AMPH_OK;
+}
+
+amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  DevState* ds = ctx->at<DevState>(l.state);
+  const int rows = ctx->rows_small;
+  launch_meta_pending(ctx->at<RowMeta>(l.meta_s), ds, st);
+  run_sals(ctx, ctx->at<float>(l.pend_h), ds->pend_tok, rows, ctx->ctx_hi);
+  launch_gather_last(ctx->at<float>(l.h1), ctx->at<float>(c.n_sal == 2 ? l.h2 : l.h1), ds, ctx->at<float>(l.last),
+                     ctx->ws + l.last_act, ctx->dtype, c.d_model, st);
+  PartialView P = project(ctx, XB_LAST, ctx->mlp_w, c.K, c.d_model, c.d_model, 2);                   // Eq. 2
+  launch_mlp_heads(P, ctx->at<float>(l.last), ctx->mlp_b, ctx->pe, ctx->at<float>(l.hp), ctx->at<float>(l.attn_o),
+                   ctx->ws + l.ao_act, ctx->dtype, c.K, c.n_sal, c.d_model, st);                      // Eq. 3-4
+  for (int a = 0; a < c.aeb_layers; ++a) {                                                            // Eq. 5
+    P = project(ctx, XB_AO, ctx->aeb_w[a], 3, c.d_model, c.d_model, c.K);
+    launch_aeb_attention(P, ctx->ws + l.aeb_act, ctx->dtype, c.K, c.n_heads, c.head_dim, st);
+    const void* wo[1] = {ctx->aeb_w[a][3]};
+    P = project(ctx, XB_AEB, wo, 1, c.d_model, c.d_model, c.K);
+    launch_resid_norm(ctx->at<float>(l.attn_o), P, 0, 1, nullptr, ctx->dtype, ctx->ws + l.ao_act, nullptr, c.rms_eps,
+                      c.K, c.d_model, st);
+  }
+  P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                               // Eq. 6
+  launch_topk_heads(P, c.vocab, c.K, c.topk, ctx->at<int>(l.topk_ids), ctx->at<float>(l.topk_vals),
+                    ctx->at<float>(l.d_logits), st);
+  launch_tree_build(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.topk_ids), nullptr, ctx->at<int>(l.tok),
+                    ctx->at<RowMeta>(l.meta_v), st);
+  amph_status rc = copy_out(ctx, out_ids, ctx->at<int>(l.topk_ids), sizeof(int) * c.K * kTopkStride);
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_vals, ctx->at<float>(l.topk_vals), sizeof(float) * c.K * kTopkStride);
+  return rc;
+}
+
+amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_argmax) {
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  const int N = ctx->tree_host.n_nodes;
+  if (tree_tokens) {
+    amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.override_tok), tree_tokens, sizeof(int) * N,
+                                                     cudaMemcpyDefault, st), "copy of tree tokens");
+    if (rc != AMPH_OK) return rc;
+    launch_tree_build(ctx->at<TreeDev>(l.tree), ctx->at<DevState>(l.state), nullptr, ctx->at<int>(l.override_tok),
+                      ctx->at<int>(l.tok), ctx->at<RowMeta>(l.meta_v), st);
+  }
+  target_forward(ctx, ctx->Mcap, ctx->ctx_hi + N);
+  target_head(ctx, ctx->Mcap);
+  return copy_out(ctx, out_argmax, ctx->at<int>(l.amax), sizeof(int) * N);
+}
+
+amph_status do_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_t* out_path, int32_t* out_next_root) {
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  DevState* ds = ctx->at<DevState>(l.state);
+  launch_accept(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.tok), ctx->at<int>(l.amax), st);
+  launch_compact(ds, ctx->at<KvView>(l.kv_tab), c.n_layers, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx,
+                 ctx->at<float>(l.hidden), ctx->at<float>(l.pend_h), c.d_model, st);
+  ctx->ctx_hi += c.K + 1;
+  amph_status rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_path, ds->path, sizeof(int) * (c.K + 1));
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_next_root, &ds->next_root, sizeof(int));
+  return rc;
+}
+
+amph_status check_capacity(amph_ctx* ctx) {
+  const int N = ctx->tree_host.n_nodes;
+  if (ctx->ctx_hi + N > ctx->cfg.max_ctx) {
+    amph_status rc = refresh_ctx_hi(ctx);
+    if (rc != AMPH_OK) return rc;
+    if (ctx->ctx_hi + N > ctx->cfg.max_ctx)
+      return fail(ctx, AMPH_ERR_CAPACITY, "ctx_len %d + %d tree nodes exceeds max_ctx %d", ctx->ctx_hi, N, ctx->cfg.max_ctx);
+  }
+  return AMPH_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+amph_status amph_workspace_bytes(const amph_config* cfg, const amph_tree* tree, size_t* kv_bytes, size_t* ws_bytes) {
+  amph_status rc = validate(cfg, tree, nullptr);
+  if (rc != AMPH_OK) return rc;
+  if (!kv_bytes || !ws_bytes) return fail(nullptr, AMPH_ERR_INVALID_ARG, "output pointers must not be NULL");
+  Layout l;
+  int Mcap;
+  make_layout(*cfg, tree->n_nodes, &l, &Mcap, kv_bytes);
+  *ws_bytes = l.total;
+  return AMPH_OK;
+}
+
+amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_dev, size_t kv_bytes, void* ws_dev,
+                      size_t ws_bytes, void* stream, amph_ctx** out) {
+  if (!out) return fail(nullptr, AMPH_ERR_INVALID_ARG, "out must not be NULL");
+  *out = nullptr;
+  TreeDev td;
+  amph_status rc = validate(cfg, tree, &td);
+  if (rc != AMPH_OK) return rc;
+  if (!kv_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "kv_dev and ws_dev must not be NULL");
+  if (((uintptr_t)kv_dev | (uintptr_t)ws_dev) & 255) return fail(nullptr, AMPH_ERR_WORKSPACE, "regions must be 256-byte aligned");
+  Layout l;
+  int Mcap;
+  size_t need_kv;
+  make_layout(*cfg, tree->n_nodes, &l, &Mcap, &need_kv);
+  if (kv_bytes < need_kv) return fail(nullptr, AMPH_ERR_WORKSPACE, "kv region: %zu bytes given, %zu needed", kv_bytes, need_kv);
+  if (ws_bytes < l.total) return fail(nullptr, AMPH_ERR_WORKSPACE, "workspace: %zu bytes given, %zu needed", ws_bytes, l.total);
+  int dev_count = 0;
+  if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count < 1) {
+    cudaGetLastError();
+    return fail(nullptr, AMPH_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  }
+  amph_ctx* ctx = new amph_ctx();
+  ctx->cfg = *cfg;
+  ctx->tree_host = td;
+  ctx->stream = (cudaStream_t)stream;
+  ctx->dtype = cfg->weight_dtype;
+  ctx->esz = cfg->weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
+  ctx->Mcap = Mcap;
+  ctx->rows_small = 16;
+  ctx->lay = l;
+  ctx->ws = (char*)ws_dev;
+  ctx->kv = (char*)kv_dev;
+  ctx->resolved = false;
+  ctx->phase = PH_CREATED;
+  ctx->ctx_hi = 0;
+  ctx->tc = nullptr;
+  const size_t half_layer = (size_t)cfg->n_heads * cfg->max_ctx * cfg->head_dim * ctx->esz;
+  ctx->kv_target.resize(cfg->n_layers);
+  char* p = ctx->kv;
+  for (int i = 0; i < cfg->n_layers; ++i) { ctx->kv_target[i].k = p; ctx->kv_target[i].v = p + half_layer; p += 2 * half_layer; }
+  for (int s = 0; s < cfg->n_sal; ++s) { ctx->kv_sal[s].k = p; ctx->kv_sal[s].v = p + half_layer; p += 2 * half_layer; }
+  cudaStream_t st = ctx->stream;
+  cudaError_t e = cudaMemsetAsync(ctx->ws, 0, l.total, st);
+  std::vector<double> inv(cfg->head_dim / 2);
+  for (int i = 0; i < cfg->head_dim / 2; ++i) inv[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.tree, &ctx->tree_host, sizeof(TreeDev), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.kv_tab, ctx->kv_target.data(), sizeof(KvView) * cfg->n_layers, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.inv_freq, inv.data(), sizeof(double) * inv.size(), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    rc = cuda_check(nullptr, e, "workspace set-up");
+    delete ctx;
+    return rc;
+  }
+  *out = ctx;
+  return AMPH_OK;
+}
+
+amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t n) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (!tensors || n < 0) return fail(ctx, AMPH_ERR_INVALID_ARG, "tensors must not be NULL");
+  for (int i = 0; i < n; ++i) {
+    const amph_tensor& t = tensors[i];
+    if (!t.name || !t.dev_ptr) return fail(ctx, AMPH_ERR_INVALID_ARG, "tensor %d: NULL name or pointer", i);
+    if (t.dtype != ctx->cfg.weight_dtype) return fail(ctx, AMPH_ERR_SHAPE, "tensor '%s': dtype %d != weight_dtype", t.name, t.dtype);
+    if (t.ndim != 1 && t.ndim != 2) return fail(ctx, AMPH_ERR_SHAPE, "tensor '%s': ndim must be 1 or 2", t.name);
+    if ((uintptr_t)t.dev_ptr & 15) return fail(ctx, AMPH_ERR_INVALID_ARG, "tensor '%s' is not 16-byte aligned", t.name);
+    TensorRec r;
+    r.ptr = t.dev_ptr;
+    r.ndim = t.ndim;
+    r.shape[0] = t.shape[0];
+    r.shape[1] = t.ndim == 2 ? t.shape[1] : 0;
+    ctx->tensors[t.name] = r;
+  }
+  ctx->resolved = false;
+  return AMPH_OK;
+}
+
+amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, int32_t* out_root) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (!prompt_ids || n < 1) return fail(ctx, AMPH_ERR_INVALID_ARG, "prompt must hold at least one token");
+  const amph_config& c = ctx->cfg;
+  for (int i = 0; i < n; ++i)
+    if (prompt_ids[i] < 0 || prompt_ids[i] >= c.vocab) return fail(ctx, AMPH_ERR_INVALID_ARG, "prompt_ids[%d] = %d is outside the vocabulary", i, prompt_ids[i]);
+  if (n + ctx->tree_host.n_nodes > c.max_ctx) return fail(ctx, AMPH_ERR_CAPACITY, "prompt of %d tokens + tree exceeds max_ctx %d", n, c.max_ctx);
+  amph_status rc = resolve(ctx);
+  if (rc != AMPH_OK) return rc;
+  if (!ctx->tc && c.weight_dtype == AMPH_DTYPE_BF16 && !(c.flags & AMPH_FLAG_NO_TENSOR_CORE)) {
+    void* xb[XB_COUNT];
+    for (int i = 0; i < XB_COUNT; ++i) xb[i] = xbuf_ptr(ctx, i);
+    const int xrows[XB_COUNT] = {ctx->Mcap, ctx->Mcap, ctx->Mcap, ctx->Mcap, 16, 16, 16};
+    const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model};
+    ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
+  }
+  const Layout& l = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  const int M = ctx->Mcap;
+  cudaMemsetAsync(ctx->ws + l.state, 0, sizeof(DevState), st);
+  for (int start = 0; start < n; start += M) {
+    const int nr = n - start < M ? n - start : M;
+    const bool last = start + nr == n;
+    rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.tok), prompt_ids + start, sizeof(int) * nr, cudaMemcpyHostToDevice, st), "prompt upload");
+    if (rc != AMPH_OK) return rc;
+    launch_meta_chain(ctx->at<RowMeta>(l.meta_v), start, nr, st);
+    target_forward(ctx, M, start + nr);
+    if (last) target_head(ctx, M);
+    const int nrs = last ? nr - 1 : nr;           // the last prompt row stays pending for the first draft
+    if (nrs > 0) {
+      rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.next_tok), prompt_ids + start + 1, sizeof(int) * nrs, cudaMemcpyHostToDevice, st), "prompt upload");
+      if (rc != AMPH_OK) return rc;
+      launch_meta_chain(ctx->at<RowMeta>(l.meta_s), start, nrs, st);
+      run_sals(ctx, ctx->at<float>(l.hidden), ctx->at<int>(l.next_tok), M, start + nrs);
+    }
+    if (last)
+      launch_prefill_tail(ctx->at<DevState>(l.state), ctx->at<int>(l.amax), nr - 1, ctx->at<float>(l.hidden),
+                          ctx->at<float>(l.pend_h), c.d_model, n, st);
+  }
+  rc = finish(ctx, "prefill");
+  if (rc != AMPH_OK) return rc;
+  rc = refresh_ctx_hi(ctx);
+  if (rc != AMPH_OK) return rc;
+  if (out_root) {
+    DevState s;
+    cudaMemcpy(&s, ctx->at<DevState>(l.state), sizeof s, cudaMemcpyDeviceToHost);
+    *out_root = s.root;
+  }
+  ctx->phase = PH_READY;
+  return AMPH_OK;
+}
+
+amph_status amph_draft(amph_ctx* ctx, int32_t* out_topk_ids, float* out_topk_vals) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->phase != PH_READY) return fail(ctx, AMPH_ERR_STATE, "amph_draft needs a prefilled sequence and no draft in flight");
+  amph_status rc = check_capacity(ctx);
+  if (rc != AMPH_OK) return rc;
+  rc = do_draft(ctx, out_topk_ids, out_topk_vals);
+  if (rc == AMPH_OK) rc = finish(ctx, "draft");
+  if (rc == AMPH_OK) ctx->phase = PH_DRAFTED;
+  return rc;
+}
+
+amph_status amph_verify_tree(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_argmax) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->phase != PH_DRAFTED) return fail(ctx, AMPH_ERR_STATE, "amph_verify_tree must follow amph_draft");
+  amph_status rc = do_verify(ctx, tree_tokens, out_argmax);
+  if (rc == AMPH_OK) rc = finish(ctx, "verify");
+  if (rc == AMPH_OK) ctx->phase = PH_VERIFIED;
+  return rc;
+}
+
+amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_t* out_path, int32_t* out_next_root) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_accept must follow amph_verify_tree");
+  amph_status rc = do_accept(ctx, out_tokens, out_n, out_path, out_next_root);
+  if (rc == AMPH_OK) rc = finish(ctx, "accept");
+  if (rc == AMPH_OK) ctx->phase = PH_READY;
+  return rc;
+}
+
+amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->phase != PH_READY) return fail(ctx, AMPH_ERR_STATE, "amph_step needs a prefilled sequence and no draft in flight");
+  amph_status rc = check_capacity(ctx);
+  if (rc != AMPH_OK) return rc;
+  rc = do_draft(ctx, nullptr, nullptr);
+  if (rc == AMPH_OK) rc = do_verify(ctx, nullptr, nullptr);
+  if (rc == AMPH_OK) rc = do_accept(ctx, out_tokens, out_n, nullptr, nullptr);
+  if (rc == AMPH_OK) rc = finish(ctx, "step");
+  return rc;
+}
+
+amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t bytes) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (!name || !dst) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and dst must not be NULL");
+  const amph_config& c = ctx->cfg;
+  const Layout& l = ctx->lay;
+  const size_t d = c.d_model, V = c.vocab, N = ctx->tree_host.n_nodes, K = c.K;
+  struct { const char* n; size_t off, size; } plain[] = {
+      {"hidden", l.hidden, 4 * N * d},   {"logits", l.logits, 4 * N * V},     {"d_logits", l.d_logits, 4 * K * V},
+      {"hp", l.hp, 4 * K * d},           {"attn_o", l.attn_o, 4 * K * d},     {"sal_h", l.last, 4 * 2 * d},
+      {"tree_tokens", l.tok, 4 * N},     {"argmax", l.amax, 4 * N},
+  };
+  for (auto& p : plain) {
+    if (strcmp(name, p.n) == 0) {
+      if (bytes > p.size) return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' holds %zu bytes, %zu requested", name, p.size, bytes);
+      return copy_out(ctx, dst, ctx->ws + p.off, bytes);
+    }
+  }
+  // cache exports: "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v", optional "@row0" suffix
+  std::string nm(name);
+  int row0 = 0;
+  const size_t at = nm.find('@');
+  if (at != std::string::npos) { row0 = atoi(nm.c_str() + at + 1); nm = nm.substr(0, at); }
+  KvView kv = {nullptr, nullptr};
+  int which = -1, idx = -1;
+  char kvc = 0;
+  if (sscanf(nm.c_str(), "kv.%c.%d", &kvc, &idx) == 2 && idx >= 0 && idx < c.n_layers) kv = ctx->kv_target[idx];
+  else if (sscanf(nm.c_str(), "sal%d.%c", &idx, &kvc) == 2 && idx >= 1 && idx <= c.n_sal) kv = ctx->kv_sal[idx - 1];
+  if (kvc == 'k') which = 0;
+  if (kvc == 'v') which = 1;
+  if (!kv.k || which < 0) return fail(ctx, AMPH_ERR_INVALID_ARG, "unknown tensor '%s'", name);
+  const size_t rows = bytes / (4 * d);
+  if (rows * 4 * d != bytes || row0 < 0 || row0 + (int)rows > c.max_ctx)
+    return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s': bytes must be a whole number of rows inside the cache", name);
+  if (rows * d > l.partial_floats) return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s': at most %zu rows per call", name, l.partial_floats / d);
+  float* stage = ctx->at<float>(l.partial);
+  launch_kv_export(kv, which, ctx->dtype, row0, (int)rows, c.n_heads, c.head_dim, c.max_ctx, stage, ctx->stream);
+  amph_status rc = finish(ctx, "cache export");
+  if (rc != AMPH_OK) return rc;
+  return copy_out(ctx, dst, stage, bytes);
+}
+
+amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (!name || !src) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and src must not be NULL");
+  if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_set_tensor must follow amph_verify_tree");
+  size_t off;
+  if (strcmp(name, "tree_tokens") == 0) off = ctx->lay.tok;
+  else if (strcmp(name, "argmax") == 0) off = ctx->lay.amax;
+  else return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' cannot be set", name);
+  if (bytes != sizeof(int) * (size_t)ctx->tree_host.n_nodes)
+    return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' takes exactly n_nodes int32 values", name);
+  return cuda_check(ctx, cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyDefault, ctx->stream), "set_tensor");
+}
+
+amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  DevState s;
+  cudaError_t e = cudaMemcpyAsync(&s, ctx->at<DevState>(ctx->lay.state), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_check(ctx, e, "state read-back");
+  if (ctx->phase != PH_CREATED) ctx->ctx_hi = s.C;
+  if (ctx_len) *ctx_len = s.C;
+  if (root) *root = s.root;
+  if (n_pending) *n_pending = s.n_pending;
+  if (s.err) return fail(ctx, s.err, "a device-side wait gave up (code %d)", s.err);
+  return AMPH_OK;
+}
+
+amph_status amph_reset(amph_ctx* ctx) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, sizeof(DevState), ctx->stream);
+  ctx->phase = PH_CREATED;
+  ctx->ctx_hi = 0;
+  return cuda_check(ctx, e, "reset");
+}
+
+void amph_destroy(amph_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->tc) tc_gemm_destroy(ctx->tc);
+  delete ctx;
+}
+
+const char* amph_last_error(const amph_ctx* ctx) { return ctx ? ctx->err.c_str() : g_last_error.c_str(); }
+
+}  // extern "C"
