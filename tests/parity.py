@@ -1,0 +1,165 @@
+"""Step-by-step comparison of the CUDA library with the CPU oracle on the same seeded inputs.
+
+Protocol (per step): both sides draft from their own state; the drafted top-k lists are
+compared; the oracle's tree tokens (drafted, or with a planted path) are handed to
+amph_verify_tree so both sides verify the same tokens; logits / hidden rows are compared
+within tolerance; integer outputs (argmax, accepted path, emitted tokens, next root,
+compacted cache rows) must be identical wherever the oracle's own decision has a margin
+larger than the floating-point tolerance.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import torch
+
+import inputs
+from oracle import amphista_oracle as ao
+
+
+@dataclass
+class Report:
+    steps: int = 0
+    max_logit_err: float = 0.0
+    max_hidden_err: float = 0.0
+    max_dlogit_err: float = 0.0
+    max_kv_err: float = 0.0
+    topk_tie_swaps: int = 0
+    argmax_near_ties: int = 0
+    gated_steps: int = 0
+    accepted: List[int] = field(default_factory=list)
+
+
+def rel_err(g: torch.Tensor, o: torch.Tensor) -> float:
+    """max |g - o| / max(1, max |o|)"""
+    o = o.to(torch.float64)
+    return float((g.to(torch.float64).cpu() - o).abs().max() / max(1.0, float(o.abs().max())))
+
+
+def plant(t: ao.TreeTables, future: List[int], leaf: int) -> List[int]:
+    ov = [-1] * t.n_nodes
+    for i, n in enumerate(t.ancestors[leaf]):
+        if i > 0 and i - 1 < len(future):
+            ov[n] = future[i - 1]
+    return ov
+
+
+def compare_topk(shape, g_ids, g_vals, o_dlogits, tie_tol, rep: Report):
+    for k in range(shape.K):
+        c = shape.topk[k]
+        row = o_dlogits[k].to(torch.float64)
+        o_ids, _ = ao.topk_desc(row, c)
+        gi = [int(v) for v in g_ids[k, :c].tolist()]
+        assert len(set(gi)) == c, f"head {k}: duplicate candidates {gi}"
+        kth = float(row[o_ids[-1]])
+        for pos, (a, b) in enumerate(zip(gi, o_ids)):
+            if a != b:
+                # only allowed when the oracle's own values are within the tie tolerance
+                assert abs(float(row[a]) - float(row[b])) <= tie_tol, \
+                    f"head {k} rank {pos}: gpu id {a} ({float(row[a]):.6f}) vs oracle id {b} ({float(row[b]):.6f})"
+                rep.topk_tie_swaps += 1
+        for a in set(gi) - set(o_ids):
+            assert float(row[a]) >= kth - tie_tol
+        gv = g_vals[k, :c].to(torch.float64).cpu()
+        ov = torch.tensor([float(row[i]) for i in gi], dtype=torch.float64)
+        assert float((gv - ov).abs().max()) <= max(tie_tol, 1e-6) * 40 + 1e-9
+
+
+def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int, tol: float,
+               tie_tol: float, planted: bool, kv_check_layers=(0, -1)) -> Report:
+    """model: paper_2406_13170_b200.Amphista.  Returns the error report; raises on a mismatch."""
+    dev = model.device
+    t = ao.tree_tables(topo.parent, topo.depth, topo.rank)
+    N, K, d, V = t.n_nodes, shape.K, shape.d_model, shape.vocab
+    rep = Report()
+    st = orc.prefill(prompt)
+    root = model.prefill(prompt)
+    assert root == st.root, f"prefill root {root} vs oracle {st.root}"
+    future = orc.greedy_ar(prompt, steps * (K + 1) + K + 2) if planted else None
+    emitted_total: List[int] = []
+    g_ids = torch.zeros(K, 16, dtype=torch.int32, device=dev)
+    g_vals = torch.zeros(K, 16, dtype=torch.float32, device=dev)
+    g_amax = torch.zeros(N, dtype=torch.int32, device=dev)
+    g_tok = torch.zeros(K + 1, dtype=torch.int32, device=dev)
+    g_path = torch.zeros(K + 1, dtype=torch.int32, device=dev)
+    g_n = torch.zeros(1, dtype=torch.int32, device=dev)
+    g_next = torch.zeros(1, dtype=torch.int32, device=dev)
+    margin = 4.0 * tol
+    for i in range(steps):
+        C0 = st.C
+        assert model.get_state()[0] == C0
+        ov = None
+        if planted:
+            leaf = t.leaves[i % len(t.leaves)]
+            ov = plant(t, future[len(emitted_total) + 1: len(emitted_total) + 1 + t.depth[leaf]], leaf)
+        taps = {}
+        emitted = orc.step(st, t, ov, taps)
+        # ---- draft
+        model.draft(g_ids, g_vals)
+        torch.cuda.synchronize(dev)
+        g_dl = model.get_tensor("d_logits", (K, V))
+        scale = max(1.0, float(taps["d_logits"].abs().max()))
+        rep.max_dlogit_err = max(rep.max_dlogit_err, rel_err(g_dl, taps["d_logits"]))
+        assert rel_err(g_dl, taps["d_logits"]) <= tol, f"step {i}: draft logits off by {rel_err(g_dl, taps['d_logits'])}"
+        assert rel_err(model.get_tensor("hp", (K, d)), taps["Hp"]) <= tol
+        assert rel_err(model.get_tensor("attn_o", (K, d)), taps["attn_o"]) <= tol
+        sal_h = model.get_tensor("sal_h", (2, d))
+        assert rel_err(sal_h[0], taps["h1"]) <= tol and rel_err(sal_h[1], taps["h2"]) <= tol
+        compare_topk(shape, g_ids, g_vals, taps["d_logits"], tie_tol * scale, rep)
+        # ---- verify the oracle's tree tokens
+        toks = torch.tensor(taps["toks"], dtype=torch.int32, device=dev)
+        model.verify_tree(toks, g_amax)
+        torch.cuda.synchronize(dev)
+        assert model.get_tensor("tree_tokens", (N,), torch.int32).tolist() == taps["toks"]
+        g_logits = model.get_tensor("logits", (N, V))
+        g_hidden = model.get_tensor("hidden", (N, d))
+        le, he = rel_err(g_logits, taps["logits"]), rel_err(g_hidden, taps["hid"])
+        rep.max_logit_err, rep.max_hidden_err = max(rep.max_logit_err, le), max(rep.max_hidden_err, he)
+        assert le <= tol, f"step {i}: logits off by {le}"
+        assert he <= tol, f"step {i}: hidden off by {he}"
+        lscale = max(1.0, float(taps["logits"].abs().max()))
+        top2 = torch.topk(taps["logits"].to(torch.float64), 2, dim=1).values
+        gaps = (top2[:, 0] - top2[:, 1])
+        safe = gaps > margin * lscale
+        ga = g_amax.tolist()
+        for n in range(N):
+            if bool(safe[n]):
+                assert ga[n] == taps["amax"][n], f"step {i} node {n}: argmax {ga[n]} vs {taps['amax'][n]}"
+            else:
+                rep.argmax_near_ties += 1
+        # ---- accept.  The acceptance kernel itself is integer logic: fed the oracle's argmax it must
+        # reproduce the oracle bit for bit, whatever the floating-point margins were.
+        all_safe = bool(safe.all())
+        if not all_safe:
+            rep.gated_steps += 1
+            model.set_tensor("argmax", torch.tensor(taps["amax"], dtype=torch.int32, device=dev))
+        model.accept(g_tok, g_n, g_path, g_next)
+        torch.cuda.synchronize(dev)
+        L = int(g_n[0])
+        assert L == taps["L"], f"step {i}: accepted {L} vs oracle {taps['L']}"
+        assert g_path[:L].tolist() == taps["path"]
+        assert g_tok[:L].tolist() == emitted
+        assert int(g_next[0]) == taps["next_root"]
+        C1, groot, npend = model.get_state()
+        assert (C1, groot, npend) == (st.C, st.root, L)
+        # ---- compacted cache rows of this step
+        for l in sorted(set(x % shape.n_layers for x in kv_check_layers)):
+            for which, cache in (("k", st.kv[l].k), ("v", st.kv[l].v)):
+                rows = model.get_tensor(f"kv.{which}.{l}@{C0}", (L, d))
+                ref = torch.stack(cache[C0:C0 + L])
+                e = rel_err(rows, ref)
+                rep.max_kv_err = max(rep.max_kv_err, e)
+                assert e <= tol, f"step {i}: layer {l} {which} cache rows off by {e}"
+        emitted_total += emitted
+        rep.accepted.append(L)
+        rep.steps += 1
+    # adaptation-layer caches cover every position committed before the last step
+    for s in range(shape.n_sal):
+        n_rows = len(st.sal_kv[s].k)
+        for which, cache in (("k", st.sal_kv[s].k), ("v", st.sal_kv[s].v)):
+            rows = model.get_tensor(f"sal{s+1}.{which}", (n_rows, d))
+            e = rel_err(rows, torch.stack(cache))
+            rep.max_kv_err = max(rep.max_kv_err, e)
+            assert e <= tol, f"stage {s+1} {which} cache off by {e}"
+    return rep

@@ -1,0 +1,50 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI."""
+import pytest
+import torch
+
+import inputs
+from inputs.configs import ModelShape
+from oracle import amphista_oracle as ao
+from tests.parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4      # fp32 kernels against the float64 oracle
+TOL_BF16 = 2e-2     # bf16 weights / activations, fp32 accumulation, against the oracle
+TIE_F32 = 1e-5
+TIE_BF16 = 1e-3
+
+
+def _setup(shape, topo, flags=0, max_ctx=None):
+    from paper_2406_13170_b200 import Amphista
+    w_cpu = inputs.make_weights(shape, seed=0)
+    w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
+    for k in ("tok_emb", "layers.0.wq", "draft.lm_head.1"):
+        assert torch.equal(w_cpu[k], w_gpu[k].cpu()), "input generator must be device independent"
+    model = Amphista(shape, topo, w_gpu, max_ctx=max_ctx, flags=flags)
+    orc = ao.Oracle(shape, w_cpu, dtype=torch.float64)
+    return model, orc
+
+
+@pytest.mark.parametrize("planted", [False, True], ids=["natural", "planted"])
+def test_tiny_fp32_eight_steps(planted):
+    shape = inputs.get_shape("tiny")
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    model, orc = _setup(shape, topo)
+    prompt = inputs.make_prompt(shape).tolist()
+    rep = run_parity(model, orc, shape, topo, prompt, shape.steps, TOL_F32, TIE_F32, planted)
+    print(rep)
+    assert rep.steps == shape.steps
+    if planted:
+        assert max(rep.accepted) >= 3
+    model.close()
+
+
+def test_tiny_depth4_tree_and_ragged_prompt():
+    shape = inputs.get_shape("tiny").with_(n_nodes=15, prompt_len=37, topk=(2, 2, 1, 1))
+    topo = inputs.full_tree([2, 2, 1, 1])
+    model, orc = _setup(shape, topo)
+    prompt = inputs.make_prompt(shape).tolist()
+    rep = run_parity(model, orc, shape, topo, prompt, 5, TOL_F32, TIE_F32, True)
+    assert max(rep.accepted) == 5
+    model.close()
