@@ -182,6 +182,15 @@ amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, si
  * device-side errors (AMPH_ERR_TIMEOUT). */
 amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending);
 
+/* Per-kernel timing of the projections (the weight-streaming kernels that dominate a step).
+ * Between amph_profile_begin and amph_profile_end every projection launch is bracketed by CUDA
+ * events on the context's stream.  amph_profile_end synchronises the stream and reports, summed over
+ * the bracketed launches: device time in milliseconds, number of launches, and weight bytes streamed
+ * (each weight matrix counted once per launch).  HOST output pointers, each may be NULL.  At most
+ * 16384 launches are recorded per begin / end pair; later ones run unrecorded. */
+amph_status amph_profile_begin(amph_ctx* ctx);
+amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launches, int64_t* proj_weight_bytes);
+
 /* Forgets the sequence (caches are logically emptied); weights stay registered. */
 amph_status amph_reset(amph_ctx* ctx);
 

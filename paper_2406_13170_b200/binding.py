@@ -23,7 +23,7 @@ STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
 EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
-           "amph_get_state",
+           "amph_get_state", "amph_profile_begin", "amph_profile_end",
            "amph_reset", "amph_destroy", "amph_last_error"]
 
 
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
         L.amph_get_tensor.argtypes = [vp, C.c_char_p, vp, C.c_size_t]
         L.amph_set_tensor.argtypes = [vp, C.c_char_p, vp, C.c_size_t]
         L.amph_get_state.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.amph_profile_begin.argtypes = [vp]
+        L.amph_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.amph_reset.argtypes = [vp]
         L.amph_destroy.argtypes = [vp]
         L.amph_destroy.restype = None
@@ -216,6 +218,15 @@ class Amphista:
         with torch.cuda.device(self.device):
             self._check(self.L.amph_get_state(self.ctx, C.byref(a), C.byref(b), C.byref(c)), self.ctx)
         return a.value, b.value, c.value
+
+    def profile_begin(self) -> None:
+        self._check(self.L.amph_profile_begin(self.ctx), self.ctx)
+
+    def profile_end(self):
+        ms, n, by = C.c_double(), C.c_int64(), C.c_int64()
+        with torch.cuda.device(self.device):
+            self._check(self.L.amph_profile_end(self.ctx, C.byref(ms), C.byref(n), C.byref(by)), self.ctx)
+        return ms.value, n.value, by.value
 
     def reset(self) -> None:
         self._check(self.L.amph_reset(self.ctx), self.ctx)

@@ -75,6 +75,10 @@ struct amph_ctx {
   int ctx_hi;               // host-side upper bound of the committed length
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
+  bool prof_on = false;     // bracket projection launches with events (amph_profile_begin / end)
+  std::vector<cudaEvent_t> prof_ev;
+  size_t prof_used = 0;
+  int64_t prof_bytes = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -274,7 +278,21 @@ void* xbuf_ptr(amph_ctx* ctx, int xb) {
   return ctx->ws + off[xb];
 }
 
+PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows);
+
 PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
+  const bool rec = ctx->prof_on && ctx->prof_used + 2 <= ctx->prof_ev.size();
+  if (rec) cudaEventRecord(ctx->prof_ev[ctx->prof_used], ctx->stream);
+  PartialView pv = project_impl(ctx, xb, w, n_seg, out, in, rows);
+  if (rec) {
+    cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], ctx->stream);
+    ctx->prof_used += 2;
+    ctx->prof_bytes += (int64_t)n_seg * out * in * (int64_t)ctx->esz;
+  }
+  return pv;
+}
+
+PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
   float* P = ctx->at<float>(ctx->lay.partial);
   PartialView pv;
   if (ctx->tc) {
@@ -720,6 +738,39 @@ amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32
   return AMPH_OK;
 }
 
+amph_status amph_profile_begin(amph_ctx* ctx) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->prof_ev.empty()) {
+    ctx->prof_ev.resize(2 * 16384);
+    for (auto& e : ctx->prof_ev)
+      if (cudaEventCreate(&e) != cudaSuccess) {
+        ctx->prof_ev.clear();
+        return cuda_check(ctx, cudaGetLastError(), "event creation");
+      }
+  }
+  ctx->prof_used = 0;
+  ctx->prof_bytes = 0;
+  ctx->prof_on = true;
+  return AMPH_OK;
+}
+
+amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launches, int64_t* proj_weight_bytes) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (!ctx->prof_on) return fail(ctx, AMPH_ERR_STATE, "amph_profile_end without amph_profile_begin");
+  ctx->prof_on = false;
+  amph_status rc = cuda_check(ctx, cudaStreamSynchronize(ctx->stream), "profile synchronise");
+  if (rc != AMPH_OK) return rc;
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < ctx->prof_used; i += 2) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, ctx->prof_ev[i], ctx->prof_ev[i + 1]) == cudaSuccess) ms += t;
+  }
+  if (proj_ms) *proj_ms = ms;
+  if (proj_launches) *proj_launches = (int64_t)(ctx->prof_used / 2);
+  if (proj_weight_bytes) *proj_weight_bytes = ctx->prof_bytes;
+  return AMPH_OK;
+}
+
 amph_status amph_reset(amph_ctx* ctx) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
   cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, sizeof(DevState), ctx->stream);
@@ -731,6 +782,7 @@ amph_status amph_reset(amph_ctx* ctx) {
 void amph_destroy(amph_ctx* ctx) {
   if (!ctx) return;
   if (ctx->tc) tc_gemm_destroy(ctx->tc);
+  for (auto& e : ctx->prof_ev) cudaEventDestroy(e);
   delete ctx;
 }
 

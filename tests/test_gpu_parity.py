@@ -9,7 +9,7 @@ from tests.parity import run_parity
 
 pytestmark = pytest.mark.gpu
 
-TOL_F32 = 1e-4      # fp32 kernels against the float64 oracle
+TOL_F32 = 1e-5      # fp32 kernels against the float64 oracle
 TOL_BF16 = 2e-2     # bf16 weights / activations, fp32 accumulation, against the oracle
 TIE_F32 = 1e-5
 TIE_BF16 = 1e-3
@@ -47,4 +47,21 @@ def test_tiny_depth4_tree_and_ragged_prompt():
     prompt = inputs.make_prompt(shape).tolist()
     rep = run_parity(model, orc, shape, topo, prompt, 5, TOL_F32, TIE_F32, True)
     assert max(rep.accepted) == 5
+    model.close()
+
+
+@pytest.mark.parametrize("flags", [1, 0], ids=["plain-kernels", "tensor-core"])
+@pytest.mark.parametrize("planted", [False, True], ids=["natural", "planted"])
+def test_small_bf16_eight_steps(planted, flags):
+    """bf16 storage, several 128-row weight tiles, a 32-node tree, a prompt that is not a
+    multiple of the chunk size; every step compared against the float64 oracle."""
+    shape = inputs.get_shape("small_bf16")
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    model, orc = _setup(shape, topo, flags=flags)
+    prompt = inputs.make_prompt(shape).tolist()
+    rep = run_parity(model, orc, shape, topo, prompt, shape.steps, TOL_BF16, TIE_BF16, planted,
+                     kv_check_layers=(0, 1, 2))
+    print(rep)
+    if planted:
+        assert max(rep.accepted) >= 3
     model.close()
