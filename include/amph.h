@@ -191,6 +191,20 @@ amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32
 amph_status amph_profile_begin(amph_ctx* ctx);
 amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launches, int64_t* proj_weight_bytes);
 
+/* The projection primitive on its own (the weight-streaming kernel every linear map of Eq. 1-6 and
+ * of the target's layers goes through):  y[r][s*out + o] = sum_k x[r][k] * w[s][o][k]  for up to 8
+ * weight matrices w[s] ([out, in] row-major, device) that share the activation rows x
+ * ([x_rows_cap, in] row-major, device, same dtype as the weights; only the first `rows` are used).
+ * w: HOST array of n_seg device pointers.  y: device fp32 [rows, n_seg*out].
+ * use_tensor_core != 0 selects the tcgen05 kernel (bf16 only; out % 128 == 0, in % 64 == 0,
+ * rows <= 128, x_rows_cap >= rows rounded up to 16) and fails with AMPH_ERR_SHAPE if the shape is
+ * not covered; 0 selects the plain CUDA-core kernel.  ws_dev: device scratch of ws_bytes >=
+ * 256 + 16 * 128 * n_seg * out * 4 bytes, 256-byte aligned; its first int32 is zeroed by the call and is set to
+ * AMPH_ERR_TIMEOUT if a bounded device-side wait gave up.  Stream-ordered; no context needed. */
+amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
+                         int32_t out, int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core,
+                         float* y_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* Forgets the sequence (caches are logically emptied); weights stay registered. */
 amph_status amph_reset(amph_ctx* ctx);
 

@@ -61,6 +61,12 @@ def rope(x: torch.Tensor, pos: int, n_heads: int, head_dim: int, theta: float) -
     return torch.cat([a * c - b * s, b * c + a * s], dim=1).reshape(-1)
 
 
+def linear(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """y = W x for every row of x; W is [out_features, in_features] (the projection every
+    fully connected layer, attention projection and vocabulary head of Eq. 1-6 applies)."""
+    return x @ w.T
+
+
 def silu(x: torch.Tensor) -> torch.Tensor:
     return x / (1.0 + torch.exp(-x))
 

@@ -9,4 +9,5 @@ from .binding import (  # noqa: F401
     library_path,
     make_config,
     make_tree,
+    project,
 )

@@ -23,7 +23,7 @@ STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
 EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
-           "amph_get_state", "amph_profile_begin", "amph_profile_end",
+           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_project",
            "amph_reset", "amph_destroy", "amph_last_error"]
 
 
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
         L.amph_get_state.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.amph_profile_begin.argtypes = [vp]
         L.amph_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.amph_project.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                   C.c_int32, C.c_int32, vp, vp, C.c_size_t, vp]
         L.amph_reset.argtypes = [vp]
         L.amph_destroy.argtypes = [vp]
         L.amph_destroy.restype = None
@@ -242,3 +244,25 @@ class Amphista:
             self.close()
         except Exception:
             pass
+
+
+def project(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, use_tensor_core: bool) -> torch.Tensor:
+    """amph_project: y[r][s*out + o] = sum_k x[r][k] * ws[s][o][k] for the first `rows` rows of x."""
+    L = lib()
+    n_seg = len(ws)
+    out, in_ = ws[0].shape
+    dev = x.device
+    y = torch.empty(rows, n_seg * out, dtype=torch.float32, device=dev)
+    scratch = torch.empty(256 + 16 * 128 * n_seg * out * 4, dtype=torch.uint8, device=dev)
+    arr = (C.c_void_p * n_seg)(*[w.data_ptr() for w in ws])
+    dt = AMPH_DTYPE_F32 if x.dtype == torch.float32 else AMPH_DTYPE_BF16
+    with torch.cuda.device(dev):
+        rc = L.amph_project(_ptr(x), x.shape[0], arr, n_seg, out, in_, rows, dt, int(use_tensor_core), _ptr(y),
+                            _ptr(scratch), scratch.numel(), C.c_void_p(torch.cuda.current_stream(dev).cuda_stream))
+        if rc != 0:
+            raise AmphError(rc, L.amph_last_error(None).decode())
+        torch.cuda.synchronize(dev)
+    err = int(scratch[:4].view(torch.int32)[0])
+    if err:
+        raise AmphError(err, "a bounded device-side wait gave up")
+    return y

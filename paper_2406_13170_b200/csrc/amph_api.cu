@@ -771,6 +771,49 @@ amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launc
   return AMPH_OK;
 }
 
+amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg, int32_t out,
+                         int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core, float* y_dev, void* ws_dev,
+                         size_t ws_bytes, void* stream) {
+  if (!x_dev || !w || !y_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "NULL pointer");
+  if (n_seg < 1 || n_seg > kMaxK || out < 1 || in < 8 || rows < 1 || rows > kMaxRows || x_rows_cap < rows)
+    return fail(nullptr, AMPH_ERR_SHAPE, "bad projection shape");
+  if (dtype != AMPH_DTYPE_F32 && dtype != AMPH_DTYPE_BF16) return fail(nullptr, AMPH_ERR_SHAPE, "unknown dtype");
+  if (in % (dtype == AMPH_DTYPE_F32 ? 4 : 8)) return fail(nullptr, AMPH_ERR_SHAPE, "in must be a multiple of 16 bytes");
+  const size_t ld = (size_t)n_seg * out;
+  const size_t need = 256 + (size_t)16 * 128 * ld * 4;
+  if (ws_bytes < need || ((uintptr_t)ws_dev & 255)) return fail(nullptr, AMPH_ERR_WORKSPACE, "scratch: %zu bytes needed, 256-byte aligned", need);
+  cudaStream_t st = (cudaStream_t)stream;
+  int* err = (int*)ws_dev;
+  float* P = (float*)((char*)ws_dev + 256);
+  const size_t p_floats = (ws_bytes - 256) / 4;
+  cudaMemsetAsync(err, 0, sizeof(int), st);
+  PartialView pv;
+  pv.p = P;
+  pv.ld = (int)ld;
+  if (use_tensor_core) {
+    if (dtype != AMPH_DTYPE_BF16) return fail(nullptr, AMPH_ERR_SHAPE, "the tensor-core kernel takes bf16 only");
+    void* xb[1] = {const_cast<void*>(x_dev)};
+    const int xr[1] = {x_rows_cap}, xc[1] = {in};
+    TcGemm* g = tc_gemm_create(xb, xr, xc, 1, err);
+    if (!g) return fail(nullptr, AMPH_ERR_CUDA, "tensor-map encoder unavailable or not an sm_100 device");
+    int splits = 0;
+    size_t stride = 0;
+    const bool ok = tc_gemm_launch(g, 0, w, n_seg, out, in, rows, P, p_floats, &splits, &stride, st);
+    tc_gemm_destroy(g);
+    if (!ok) return fail(nullptr, AMPH_ERR_SHAPE, "shape not covered by the tensor-core kernel");
+    pv.splits = splits;
+    pv.split_stride = stride;
+  } else {
+    GemmSeg segs[kMaxK];
+    for (int s = 0; s < n_seg; ++s) segs[s].w = w[s];
+    launch_gemm_generic(x_dev, in, segs, n_seg, out, in, P, (int)ld, rows, dtype, st);
+    pv.splits = 1;
+    pv.split_stride = 0;
+  }
+  launch_reduce_partials(pv, y_dev, rows, (int)ld, st);
+  return cuda_check(nullptr, cudaGetLastError(), "projection");
+}
+
 amph_status amph_reset(amph_ctx* ctx) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
   cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, sizeof(DevState), ctx->stream);

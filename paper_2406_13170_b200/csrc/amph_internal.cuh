@@ -124,6 +124,7 @@ void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, co
 void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st);
 void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
                     int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st);
+void launch_reduce_partials(PartialView P, float* y, int rows, int cols, cudaStream_t st);
 void launch_kv_export(KvView kv, int which, int dtype, int row0, int rows, int n_heads, int head_dim, int max_ctx,
                       float* dst, cudaStream_t st);
 void launch_prefill_tail(DevState* s, const int* amax, int last_row, const float* hidden, float* pend_h,

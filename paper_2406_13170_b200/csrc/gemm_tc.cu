@@ -1,7 +1,352 @@
+// Skinny bf16 projection on the 5th-generation tensor cores:  Y^T[out][rows] = W[out][in] . X^T.
+//
+// The weight matrix is the 128-row MMA operand A (K-major, streamed once from HBM by TMA), the few
+// activation rows are operand B (N = 16..128 rows, K-major, re-read from L2), the fp32 accumulator
+// lives in tensor memory.  One CTA owns one 128-row weight tile and one K-range (split-K); partial
+// sums go to global memory as P[split][row][feature] and are reduced, in a fixed order, by the
+// kernel that consumes them.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the TMEM
+// allocation), warps 2-5 = epilogue (TMEM -> registers -> global).  Every barrier wait is bounded:
+// if one gives up the CTA sets *err_flag, drains its own copies and exits cleanly.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <map>
+#include <tuple>
+
+#include "amph.h"
 #include "gemm_tc.cuh"
+
 namespace amph {
-struct TcGemm {};
-TcGemm* tc_gemm_create(void* const*, const int*, const int*, int, int*) { return nullptr; }
-bool tc_gemm_launch(TcGemm*, int, const void* const*, int, int, int, int, float*, size_t, int*, size_t*, cudaStream_t) { return false; }
-void tc_gemm_destroy(TcGemm* g) { delete g; }
+
+namespace {
+
+constexpr int kTileM = 128;           // weight rows per CTA (UMMA M)
+constexpr int kTileK = 64;            // bf16 elements per 128-byte swizzle row
+constexpr int kUmmaK = 16;            // K per tcgen05.mma for 16-bit inputs
+constexpr int kMaxSeg = 8;
+constexpr int kThreads = 192;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // a barrier wait gives up after one second
+
+struct TmapPack {
+  CUtensorMap w[kMaxSeg];
+  CUtensorMap x;
+};
+
+struct TcParams {
+  float* P;
+  size_t split_stride;      // floats between splits
+  int ld;                   // floats per row of P
+  int tiles_per_seg;        // out / 128
+  int kblocks;              // in / 64
+  int splits;
+  int nt;                   // activation rows in the MMA (multiple of 16)
+  int rows;                 // live rows (only these are stored)
+  int stages;
+  int* err_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; returns false (and raises the shared abort flag) if the phase never completes or
+// another role already gave up.
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = now_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try(bar, parity)) return true;
+    if ((i & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > kWaitLimitNs) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                                // leading-dimension offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                      // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                                // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = nt.
+__device__ __forceinline__ uint32_t umma_idesc(int nt) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads)
+tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[8];
+  __shared__ __align__(8) uint64_t empty_bar[8];
+  __shared__ __align__(8) uint64_t accum_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  const int seg = tile / prm.tiles_per_seg;
+  const int row0 = (tile - seg * prm.tiles_per_seg) * kTileM;       // first weight row of this tile
+  const int kb_lo = (int)((long long)split * prm.kblocks / prm.splits);
+  const int kb_hi = (int)((long long)(split + 1) * prm.kblocks / prm.splits);
+  const int nkb = kb_hi - kb_lo;
+  const int nt = prm.nt, stages = prm.stages;
+  const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
+  const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < nt) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {                                   // TMEM allocation belongs to the MMA warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_base_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      const CUtensorMap* wmap = &maps.w[seg];
+      asm volatile("prefetch.tensormap [%0];" ::"l"(wmap) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x) : "memory");
+      int issued = 0;
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % stages, round = i / stages;
+        if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag)) break;
+        uint8_t* a = smem + (size_t)s * stage_bytes;
+        mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+        tma_load_2d(a, wmap, (kb_lo + i) * kTileK, row0, &full_bar[s]);
+        tma_load_2d(a + a_bytes, &maps.x, (kb_lo + i) * kTileK, 0, &full_bar[s]);
+        issued = i + 1;
+      }
+      if (abort_flag) {                              // drain: let every copy this thread issued land
+        const int first = issued > stages ? issued - stages : 0;
+        for (int i = first; i < issued; ++i) {
+          const int s = i % stages, round = i / stages;
+          const unsigned long long t0 = now_ns();
+          while (!mbar_try(&full_bar[s], round & 1) && now_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc(nt);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        const int s = i % stages, round = i / stages;
+        ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + a_bytes);
+#pragma unroll
+        for (int k = 0; k < kTileK / kUmmaK; ++k)      // +32 bytes (2 x 16 B) per K step inside the swizzle row
+          umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | k) ? 1u : 0u);
+        umma_commit(&empty_bar[s]);                    // frees the stage once these MMAs have read it
+      }
+      if (ok) umma_commit(&accum_bar);
+    }
+  } else {
+    // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    const int quarter = warp & 3;
+    const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag) : false);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int feat = seg * prm.tiles_per_seg * kTileM + row0 + quarter * 32 + lane;
+    float* out = prm.P + (size_t)split * prm.split_stride + feat;
+    for (int c0 = 0; c0 < nt; c0 += 16) {
+      if (c0 >= prm.rows) break;
+      uint32_t v[16];
+      if (ok) {
+        const uint32_t taddr = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+            : "r"(taddr)
+            : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = 0u;          // empty K-range or aborted: contribute zeros
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (c0 + j < prm.rows) out[(size_t)(c0 + j) * prm.ld] = __uint_as_float(v[j]);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
+  }
+  if (threadIdx.x == 0 && abort_flag && prm.err_flag) *prm.err_flag = AMPH_ERR_TIMEOUT;
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct TcGemm {
+  EncodeFn encode = nullptr;
+  int* err_flag = nullptr;
+  int n_x = 0;
+  void* xptr[16];
+  int xrows[16], xcols[16];
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;   // (ptr, rows, cols, box rows)
+  int sm_count = 148;
+  int max_smem = 0;
+
+  const CUtensorMap* get(const void* ptr, int rows, int cols, int box_rows) {
+    auto key = std::make_tuple(ptr, rows, cols, box_rows);
+    auto it = cache.find(key);
+    if (it != cache.end()) return &it->second;
+    CUtensorMap m;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return nullptr;
+    return &(cache[key] = m);
+  }
+};
+
+TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, int n, int* err_flag) {
+  if (n > 16) return nullptr;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  int dev = 0, major = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (major != 10) return nullptr;
+  TcGemm* g = new TcGemm();
+  g->encode = (EncodeFn)fn;
+  g->err_flag = err_flag;
+  g->n_x = n;
+  for (int i = 0; i < n; ++i) { g->xptr[i] = xbufs[i]; g->xrows[i] = xrows[i]; g->xcols[i] = xcols[i]; }
+  cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&g->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  return g;
+}
+
+bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out, int in, int rows, float* P,
+                    size_t p_floats, int* splits_out, size_t* split_stride, cudaStream_t st) {
+  if (!g || xb < 0 || xb >= g->n_x) return false;
+  if (out % kTileM || in % kTileK || n_seg < 1 || n_seg > kMaxSeg || rows < 1) return false;
+  if (g->xcols[xb] != in) return false;
+  const int nt = rows <= 16 ? 16 : (rows + 15) / 16 * 16;
+  if (nt > 128 || nt > g->xrows[xb]) return false;
+  const int tiles = n_seg * (out / kTileM), kblocks = in / kTileK;
+  const size_t ld = (size_t)n_seg * out;
+  // K-splits: fill about two CTAs per SM, keep at least four 64-wide K blocks per CTA
+  int splits = (2 * g->sm_count) / tiles;
+  if (splits > kblocks / 4) splits = kblocks / 4;
+  if (splits > 16) splits = 16;
+  while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
+  if (splits < 1) splits = 1;
+  if ((size_t)nt * ld > p_floats) return false;
+  TmapPack pack;
+  memset(&pack, 0, sizeof pack);
+  for (int s = 0; s < n_seg; ++s) {
+    if ((uintptr_t)w[s] & 15) return false;
+    const CUtensorMap* m = g->get(w[s], out, in, kTileM);
+    if (!m) return false;
+    pack.w[s] = *m;
+  }
+  const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt);
+  if (!mx) return false;
+  pack.x = *mx;
+  const uint32_t stage_bytes = kTileM * kTileK * 2 + (((uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  int stages = (int)((100 * 1024) / stage_bytes);          // <= ~100 KB per CTA: two CTAs per SM
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  TcParams prm;
+  prm.P = P;
+  prm.split_stride = (size_t)nt * ld;
+  prm.ld = (int)ld;
+  prm.tiles_per_seg = out / kTileM;
+  prm.kblocks = kblocks;
+  prm.splits = splits;
+  prm.nt = nt;
+  prm.rows = rows;
+  prm.stages = stages;
+  prm.err_flag = g->err_flag;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  tc_gemm_kernel<<<dim3(tiles, splits), kThreads, smem, st>>>(pack, prm);
+  *splits_out = splits;
+  *split_stride = prm.split_stride;
+  return true;
+}
+
+void tc_gemm_destroy(TcGemm* g) { delete g; }
+
+}  // namespace amph

@@ -772,6 +772,21 @@ void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, in
                                                                        max_ctx, hidden, pend_h, d));
 }
 
+__global__ void reduce_partials_kernel(PartialView P, float* __restrict__ y, int rows, int cols) {
+  const size_t n = (size_t)rows * cols;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / cols), c = (int)(i - (size_t)r * cols);
+    y[i] = sum_partials(P, r, c);
+  }
+}
+
+void launch_reduce_partials(PartialView P, float* y, int rows, int cols, cudaStream_t st) {
+  const size_t n = (size_t)rows * cols;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  reduce_partials_kernel<<<blocks, 256, 0, st>>>(P, y, rows, cols);
+}
+
 template <typename T>
 __global__ void kv_export_kernel(const T* __restrict__ c, int row0, int n_heads, int dh, int max_ctx,
                                  float* __restrict__ dst) {

@@ -85,7 +85,6 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
     g_path = torch.zeros(K + 1, dtype=torch.int32, device=dev)
     g_n = torch.zeros(1, dtype=torch.int32, device=dev)
     g_next = torch.zeros(1, dtype=torch.int32, device=dev)
-    margin = 4.0 * tol
     for i in range(steps):
         C0 = st.C
         assert model.get_state()[0] == C0
@@ -124,7 +123,9 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
         lscale = max(1.0, float(taps["logits"].abs().max()))
         top2 = torch.topk(taps["logits"].to(torch.float64), 2, dim=1).values
         gaps = (top2[:, 0] - top2[:, 1])
-        safe = gaps > margin * lscale
+        # a greedy choice can only flip if the oracle's top-2 gap is below twice the measured logit error
+        e_log = float((g_logits.to(torch.float64).cpu() - taps["logits"].to(torch.float64)).abs().max())
+        safe = gaps > max(2.0 * e_log, 1e-6 * lscale)
         ga = g_amax.tolist()
         for n in range(N):
             if bool(safe[n]):
