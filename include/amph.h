@@ -205,6 +205,29 @@ amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* cons
                          int32_t out, int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core,
                          float* y_dev, void* ws_dev, size_t ws_bytes, void* stream);
 
+/* (No counterpart in the paper: a packaging variant of amph_project.)
+ * The same projection for callers that cannot allocate device memory at the time of the call: for
+ * example code running after a serving engine has taken all free GPU memory into its own pool, where
+ * a cudaMalloc would fail, or a latency-critical loop that must not meet the implicit synchronisation
+ * of an allocation.  Instead of caller-provided scratch, the split-K partial sums live in a fixed
+ * array of AMPH_NOALLOC_SCRATCH_BYTES inside the library image; every GPU that loads the library
+ * holds that array until the process exits.  The call allocates nothing (no cudaMalloc / cudaFree).
+ * Arguments as for amph_project, except:
+ *   status_dev : device int32, may be NULL; zeroed by the call, set to AMPH_ERR_TIMEOUT if a bounded
+ *                device-side wait gave up (with NULL the flag is kept inside the scratch, unread);
+ *   err_msg    : HOST buffer of err_len bytes that receives a message on failure, may be NULL.
+ * Limit: 256 + (rows rounded up to 16) * n_seg * out * 4 bytes must not exceed
+ * AMPH_NOALLOC_SCRATCH_BYTES, otherwise AMPH_ERR_WORKSPACE (nothing is launched).
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before starting any stream capture.  All calls on a device share the one
+ * array, which keeps the previous call's contents (the call clears what must start at zero): calls
+ * whose kernels may overlap on the GPU (different streams, or several threads) race on it, so
+ * serialise them.  Stream-ordered; y_dev is valid once the stream has been synchronised. */
+#define AMPH_NOALLOC_SCRATCH_BYTES (16u << 20)
+amph_status amph_project_noalloc(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
+                                 int32_t out, int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core,
+                                 float* y_dev, int32_t* status_dev, void* stream, char* err_msg, size_t err_len);
+
 /* Forgets the sequence (caches are logically emptied); weights stay registered. */
 amph_status amph_reset(amph_ctx* ctx);
 

@@ -10,4 +10,5 @@ from .binding import (  # noqa: F401
     make_config,
     make_tree,
     project,
+    project_noalloc,
 )

@@ -23,7 +23,7 @@ STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
 EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
-           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_project",
+           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_project", "amph_project_noalloc",
            "amph_reset", "amph_destroy", "amph_last_error"]
 
 
@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
         L.amph_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.amph_project.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_int32, vp, vp, C.c_size_t, vp]
+        L.amph_project_noalloc.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                           C.c_int32, C.c_int32, vp, vp, vp, C.c_char_p, C.c_size_t]
         L.amph_reset.argtypes = [vp]
         L.amph_destroy.argtypes = [vp]
         L.amph_destroy.restype = None
@@ -266,3 +268,26 @@ def project(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, use_tensor_c
     if err:
         raise AmphError(err, "a bounded device-side wait gave up")
     return y
+
+
+def project_noalloc(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, use_tensor_core: bool,
+                    y: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    """amph_project_noalloc: like `project`, for callers that cannot allocate device memory when they
+    call (all free memory already belongs to someone else's pool, or an allocation's hidden
+    synchronisation is not acceptable).  The split-K scratch is a fixed array inside the library, so the
+    caller passes only inputs and the preallocated outputs `y` (fp32 [rows, n_seg*out]) and, optionally,
+    `status` (int32 [1]).  Nothing is allocated here either: no torch tensor is created.
+    Calls share the built-in scratch: do not let two of them overlap on the GPU."""
+    L = lib()
+    n_seg = len(ws)
+    out, in_ = ws[0].shape
+    dev = x.device
+    arr = (C.c_void_p * n_seg)(*[w.data_ptr() for w in ws])
+    dt = AMPH_DTYPE_F32 if x.dtype == torch.float32 else AMPH_DTYPE_BF16
+    msg = C.create_string_buffer(512)
+    with torch.cuda.device(dev):
+        rc = L.amph_project_noalloc(_ptr(x), x.shape[0], arr, n_seg, out, in_, rows, dt, int(use_tensor_core),
+                                    _ptr(y), _ptr(status), C.c_void_p(torch.cuda.current_stream(dev).cuda_stream),
+                                    msg, len(msg))
+    if rc != 0:
+        raise AmphError(rc, msg.value.decode())
