@@ -150,7 +150,9 @@ class Amphista:
         with torch.cuda.device(self.device):
             self.kv = torch.empty(kvb.value, dtype=torch.uint8, device=self.device)
             self.ws = torch.empty(wsb.value, dtype=torch.uint8, device=self.device)
-            self.stream = stream or torch.cuda.current_stream(self.device)
+            # a stream of its own: the legacy default stream cannot be captured into a CUDA graph
+            self.stream = stream or torch.cuda.Stream(self.device)
+            self.stream.wait_stream(torch.cuda.current_stream(self.device))
             self.ctx = C.c_void_p()
             self._check(self.L.amph_init(C.byref(self.cfg), C.byref(self.tree.c), _ptr(self.kv), kvb.value,
                                          _ptr(self.ws), wsb.value, C.c_void_p(self.stream.cuda_stream),
@@ -160,6 +162,13 @@ class Amphista:
         N, K = topo.n_nodes, shape.K
         self.out_tokens = torch.empty(K + 1, dtype=torch.int32, device=self.device)
         self.out_n = torch.empty(1, dtype=torch.int32, device=self.device)
+
+    def _after_torch(self) -> None:
+        """Orders the library's stream after work torch has queued on its current stream (inputs)."""
+        self.stream.wait_stream(torch.cuda.current_stream(self.device))
+
+    def synchronize(self) -> None:
+        self.stream.synchronize()
 
     def _check(self, status: int, ctx) -> None:
         if status != 0:
@@ -178,6 +187,7 @@ class Amphista:
             arr[i].ndim = t.dim()
             for j, s in enumerate(t.shape):
                 arr[i].shape[j] = s
+        self._after_torch()
         self._check(self.L.amph_load_weights(self.ctx, arr, len(weights)), self.ctx)
 
     def prefill(self, prompt: Sequence[int]) -> int:
@@ -193,6 +203,7 @@ class Amphista:
             self._check(self.L.amph_draft(self.ctx, _ptr(out_ids), _ptr(out_vals)), self.ctx)
 
     def verify_tree(self, tree_tokens: Optional[torch.Tensor] = None, out_argmax: Optional[torch.Tensor] = None) -> None:
+        self._after_torch()
         with torch.cuda.device(self.device):
             self._check(self.L.amph_verify_tree(self.ctx, _ptr(tree_tokens), _ptr(out_argmax)), self.ctx)
 
@@ -210,9 +221,11 @@ class Amphista:
         with torch.cuda.device(self.device):
             self._check(self.L.amph_get_tensor(self.ctx, name.encode(), _ptr(out), out.numel() * out.element_size()),
                         self.ctx)
+        self.stream.synchronize()
         return out
 
     def set_tensor(self, name: str, src: torch.Tensor) -> None:
+        self._after_torch()
         with torch.cuda.device(self.device):
             self._check(self.L.amph_set_tensor(self.ctx, name.encode(), _ptr(src), src.numel() * src.element_size()),
                         self.ctx)

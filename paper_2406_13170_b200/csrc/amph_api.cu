@@ -75,6 +75,9 @@ struct amph_ctx {
   int ctx_hi;               // host-side upper bound of the committed length
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
+  cudaGraphExec_t graph_exec = nullptr;   // captured draft -> verify -> accept schedule of amph_step
+  int graph_key = -1;       // attention split counts the captured grids were sized for
+  bool graph_off = false;   // capture is not possible (legacy stream, flag) or failed once
   bool prof_on = false;     // bracket projection launches with events (amph_profile_begin / end)
   std::vector<cudaEvent_t> prof_ev;
   size_t prof_used = 0;
@@ -463,12 +466,17 @@ amph_status do_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_
   launch_accept(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.tok), ctx->at<int>(l.amax), st);
   launch_compact(ds, ctx->at<KvView>(l.kv_tab), c.n_layers, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx,
                  ctx->at<float>(l.hidden), ctx->at<float>(l.pend_h), c.d_model, st);
-  ctx->ctx_hi += c.K + 1;
   amph_status rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
   if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
   if (rc == AMPH_OK) rc = copy_out(ctx, out_path, ds->path, sizeof(int) * (c.K + 1));
   if (rc == AMPH_OK) rc = copy_out(ctx, out_next_root, &ds->next_root, sizeof(int));
   return rc;
+}
+
+int attn_splits_for(const amph_ctx* ctx, int ctx_hi) {
+  int s = (ctx_hi + 127) / 128;
+  if (s > ctx->lay.attn_splits) s = ctx->lay.attn_splits;
+  return s < 1 ? 1 : s;
 }
 
 amph_status check_capacity(amph_ctx* ctx) {
@@ -574,6 +582,11 @@ amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t
     ctx->tensors[t.name] = r;
   }
   ctx->resolved = false;
+  if (ctx->graph_exec) {                       // the captured schedule holds the old pointers
+    cudaGraphExecDestroy(ctx->graph_exec);
+    ctx->graph_exec = nullptr;
+    ctx->graph_key = -1;
+  }
   return AMPH_OK;
 }
 
@@ -654,7 +667,7 @@ amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int3
   if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_accept must follow amph_verify_tree");
   amph_status rc = do_accept(ctx, out_tokens, out_n, out_path, out_next_root);
   if (rc == AMPH_OK) rc = finish(ctx, "accept");
-  if (rc == AMPH_OK) ctx->phase = PH_READY;
+  if (rc == AMPH_OK) { ctx->phase = PH_READY; ctx->ctx_hi += ctx->cfg.K + 1; }
   return rc;
 }
 
@@ -663,10 +676,46 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n) {
   if (ctx->phase != PH_READY) return fail(ctx, AMPH_ERR_STATE, "amph_step needs a prefilled sequence and no draft in flight");
   amph_status rc = check_capacity(ctx);
   if (rc != AMPH_OK) return rc;
-  rc = do_draft(ctx, nullptr, nullptr);
-  if (rc == AMPH_OK) rc = do_verify(ctx, nullptr, nullptr);
-  if (rc == AMPH_OK) rc = do_accept(ctx, out_tokens, out_n, nullptr, nullptr);
+  const amph_config& c = ctx->cfg;
+  DevState* ds = ctx->at<DevState>(ctx->lay.state);
+  const bool use_graph = !ctx->graph_off && !ctx->prof_on && !(c.flags & AMPH_FLAG_NO_GRAPH) && ctx->stream != nullptr;
+  if (use_graph) {
+    // The kernels read every length from device state; only the attention grids depend on the host's
+    // bound of the context length, so the captured schedule is reused until that grid size changes.
+    const int key = attn_splits_for(ctx, ctx->ctx_hi) * 64 + attn_splits_for(ctx, ctx->ctx_hi + ctx->tree_host.n_nodes);
+    if (!ctx->graph_exec || key != ctx->graph_key) {
+      if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+        rc = do_draft(ctx, nullptr, nullptr);
+        if (rc == AMPH_OK) rc = do_verify(ctx, nullptr, nullptr);
+        if (rc == AMPH_OK) rc = do_accept(ctx, nullptr, nullptr, nullptr, nullptr);
+        const cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+        if (rc == AMPH_OK && e == cudaSuccess && graph &&
+            cudaGraphInstantiate(&ctx->graph_exec, graph, 0) == cudaSuccess) {
+          ctx->graph_key = key;
+        } else {
+          ctx->graph_exec = nullptr;
+          ctx->graph_off = true;
+        }
+        if (graph) cudaGraphDestroy(graph);
+      } else {
+        ctx->graph_off = true;
+      }
+      cudaGetLastError();
+    }
+  }
+  if (use_graph && ctx->graph_exec) {
+    rc = cuda_check(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream), "graph launch");
+  } else {
+    rc = do_draft(ctx, nullptr, nullptr);
+    if (rc == AMPH_OK) rc = do_verify(ctx, nullptr, nullptr);
+    if (rc == AMPH_OK) rc = do_accept(ctx, nullptr, nullptr, nullptr, nullptr);
+  }
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
+  if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
   if (rc == AMPH_OK) rc = finish(ctx, "step");
+  if (rc == AMPH_OK) ctx->ctx_hi += c.K + 1;
   return rc;
 }
 
@@ -825,6 +874,7 @@ amph_status amph_reset(amph_ctx* ctx) {
 void amph_destroy(amph_ctx* ctx) {
   if (!ctx) return;
   if (ctx->tc) tc_gemm_destroy(ctx->tc);
+  if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
   for (auto& e : ctx->prof_ev) cudaEventDestroy(e);
   delete ctx;
 }

@@ -91,6 +91,9 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
                            int dtype, int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi,
                            int max_splits, cudaStream_t st);
 
+void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
+                               int head_dim, int max_ctx, int splits, cudaStream_t st);
+
 void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st);
 
 // cat[r] = [feat[r] ; tok_emb[next[r]]]   (Eq. 1's concatenation)

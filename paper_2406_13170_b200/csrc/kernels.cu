@@ -28,6 +28,32 @@ __device__ __forceinline__ float sum_partials(const PartialView& P, int row, int
   return acc;
 }
 
+__device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, int col) {
+  const float* p = P.p + (size_t)row * P.ld + col;
+  float4 acc = *reinterpret_cast<const float4*>(p);
+#pragma unroll 4
+  for (int s = 1; s < P.splits; ++s) {
+    const float4 v = *reinterpret_cast<const float4*>(p + (size_t)s * P.split_stride);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  return acc;
+}
+
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void store4(bf16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<unsigned*>(&a);
+  u.y = *reinterpret_cast<unsigned*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const bf16* p) {
+  const uint2 u = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                     __uint_as_float(u.y & 0xffff0000u));
+}
+
 __device__ __forceinline__ float block_sum(float v, float* red) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   const int w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
@@ -61,45 +87,50 @@ void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, in
 // residual update + RMSNorm (one block per row)
 // --------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode,
-                                  const T* __restrict__ gain, T* __restrict__ xn, float* __restrict__ hid,
-                                  float eps, int d) {
-  extern __shared__ float rowbuf[];
+__global__ void __launch_bounds__(1024)
+resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, const T* __restrict__ gain,
+                  T* __restrict__ xn, float* __restrict__ hid, float eps, int d) {
+  extern __shared__ __align__(16) float rowbuf[];
   __shared__ float red[32];
   const int r = blockIdx.x;
+  float* xr = x + (size_t)r * d;
   float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float v;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    float4 v;
     if (mode == 0) {
-      v = x[(size_t)r * d + c];
+      v = load4(xr + c);
     } else {
-      v = sum_partials(P, r, col_off + c);
-      if (mode == 1) v += x[(size_t)r * d + c];
-      x[(size_t)r * d + c] = v;
+      v = sum_partials4(P, r, col_off + c);
+      if (mode == 1) { const float4 o = load4(xr + c); v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+      store4(xr + c, v);
     }
-    rowbuf[c] = v;
-    ss += v * v;
+    store4(rowbuf + c, v);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   if (xn == nullptr && hid == nullptr) return;
-  if (gain == nullptr) {                       // plain cast of the updated row
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-      if (xn) xn[(size_t)r * d + c] = from_f<T>(rowbuf[c]);
-      if (hid) hid[(size_t)r * d + c] = rowbuf[c];
+  if (gain == nullptr) {                       // plain cast of the updated row (each thread re-reads its own chunk)
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+      const float4 v = load4(rowbuf + c);
+      if (xn) store4(xn + (size_t)r * d + c, v);
+      if (hid) store4(hid + (size_t)r * d + c, v);
     }
     return;
   }
   const float tot = block_sum(ss, red);
   const float inv = 1.0f / sqrtf(tot / (float)d + eps);
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float n = to_f(gain[c]) * (rowbuf[c] * inv);
-    if (xn) xn[(size_t)r * d + c] = from_f<T>(n);
-    if (hid) hid[(size_t)r * d + c] = n;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    const float4 v = load4(rowbuf + c), g = load4(gain + c);
+    const float4 n = make_float4(g.x * (v.x * inv), g.y * (v.y * inv), g.z * (v.z * inv), g.w * (v.w * inv));
+    if (xn) store4(xn + (size_t)r * d + c, n);
+    if (hid) store4(hid + (size_t)r * d + c, n);
   }
 }
 
 void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
                        void* xn, float* hid, float eps, int rows, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, resid_norm_kernel<T><<<rows, 256, d * sizeof(float), st>>>(
+  int threads = (d / 4 + 31) / 32 * 32;
+  if (threads > 1024) threads = 1024;
+  AMPH_DISPATCH(dtype, resid_norm_kernel<T><<<rows, threads, d * sizeof(float), st>>>(
                            x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d));
 }
 
@@ -126,36 +157,45 @@ void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* tabl
 // q / k rotation, KV-cache write (one block per row)
 // --------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta,
-                                const float2* __restrict__ rope, T* __restrict__ q, T* __restrict__ kc,
-                                T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
+__global__ void __launch_bounds__(1024)
+qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* __restrict__ rope, T* __restrict__ q,
+                T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
   const int r = blockIdx.x;
-  const int half = dh >> 1, d = n_heads * dh;
+  const int half = dh >> 1, d = n_heads * dh, quads = half >> 2;
   const bool live = r < meta->n_rows;
   const int slot = meta->slot[r];
   const bool store = live && slot >= 0 && slot < max_ctx;
-  for (int idx = threadIdx.x; idx < n_heads * half; idx += blockDim.x) {
-    const int h = idx / half, i = idx - h * half;
-    const float2 cs = rope[r * half + i];
+  for (int idx = threadIdx.x; idx < n_heads * quads; idx += blockDim.x) {
+    const int h = idx / quads, i = (idx - h * quads) * 4;          // four rotation pairs (i..i+3, i+half..)
+    const float4 cs0 = *reinterpret_cast<const float4*>(rope + r * half + i);       // (c0,s0,c1,s1)
+    const float4 cs1 = *reinterpret_cast<const float4*>(rope + r * half + i + 2);   // (c2,s2,c3,s3)
     const int c0 = h * dh + i, c1 = c0 + half;
-    const float q0 = sum_partials(P, r, c0), q1 = sum_partials(P, r, c1);
-    q[(size_t)r * d + c0] = from_f<T>(q0 * cs.x - q1 * cs.y);
-    q[(size_t)r * d + c1] = from_f<T>(q1 * cs.x + q0 * cs.y);
+    {
+      const float4 a = sum_partials4(P, r, c0), b = sum_partials4(P, r, c1);
+      store4(q + (size_t)r * d + c0, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
+                                                 a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
+      store4(q + (size_t)r * d + c1, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
+                                                 b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
+    }
     if (store) {
-      const float k0 = sum_partials(P, r, d + c0), k1 = sum_partials(P, r, d + c1);
+      const float4 a = sum_partials4(P, r, d + c0), b = sum_partials4(P, r, d + c1);
       const size_t o = ((size_t)h * max_ctx + slot) * dh + i;
-      kc[o] = from_f<T>(k0 * cs.x - k1 * cs.y);
-      kc[o + half] = from_f<T>(k1 * cs.x + k0 * cs.y);
-      vc[o] = from_f<T>(sum_partials(P, r, 2 * d + c0));
-      vc[o + half] = from_f<T>(sum_partials(P, r, 2 * d + c1));
+      store4(kc + o, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
+                                 a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
+      store4(kc + o + half, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
+                                        b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
+      store4(vc + o, sum_partials4(P, r, 2 * d + c0));
+      store4(vc + o + half, sum_partials4(P, r, 2 * d + c1));
     }
   }
 }
 
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv, int dtype,
                      int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, qkv_rope_kernel<T><<<rows, 256, 0, st>>>(P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
-                                                                n_heads, head_dim, max_ctx));
+  int threads = (n_heads * head_dim / 8 + 31) / 32 * 32;
+  if (threads > 1024) threads = 1024;
+  AMPH_DISPATCH(dtype, qkv_rope_kernel<T><<<rows, threads, 0, st>>>(P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
+                                                                    n_heads, head_dim, max_ctx));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -334,6 +374,12 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
   int splits = (ctx_hi + 127) / 128;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
+  if (dtype == AMPH_DTYPE_BF16) {                    // tensor-core path; the kernel below serves fp32 caches
+    launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st);
+    attn_combine_kernel<bf16><<<dim3(rows, n_heads), head_dim < 128 ? 64 : 128, 0, st>>>(sc.o, sc.ml, (bf16*)out, splits,
+                                                                                        rows, n_heads, head_dim);
+    return;
+  }
   if (head_dim == 64) {
     AMPH_DISPATCH(dtype, (tree_attention_t<T, 64>(q, kv, meta, sc, out, rows, n_heads, max_ctx, splits, st)));
   } else {
