@@ -53,6 +53,31 @@ struct DevState {
   int out_tok[16];
 };
 
+// Programmatic dependent launch.  Every kernel of the step is launched with the attribute below, so it
+// may become resident before its predecessor in the stream has finished; it must call pdl_wait() before
+// touching anything the predecessor writes.  pdl_launch_dependents() lets the successor start launching.
+// Rule used here: weight-streaming projections trigger at once, prefetch weights, then wait; every other
+// kernel waits first and triggers right after, so at most two consecutive kernels ever overlap.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... P, typename... A>
+inline cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+#endif
+
 struct KvView {             // one layer's cache: K and V as [n_heads][max_ctx][head_dim]
   void* k;
   void* v;

@@ -68,6 +68,8 @@ __global__ void __launch_bounds__(kThreads)
 tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, const bf16* __restrict__ vc,
                      const RowMeta* __restrict__ meta, float* __restrict__ po, float* __restrict__ pml,
                      int rows_cap, int n_heads, int max_ctx) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int KS = DH / 16;                        // k-steps over the head dimension
   constexpr int NT = DH / 8;                         // 8-wide output tiles
   extern __shared__ __align__(128) unsigned char sm_raw[];
@@ -245,7 +247,7 @@ void launch_t(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int
   const size_t smem = sizeof(bf16) * (kRows * DH + 4 * kKeys * DH);
   cudaFuncSetAttribute(tree_attn_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid(n_heads, splits, (rows + kRows - 1) / kRows);
-  tree_attn_mma_kernel<DH><<<grid, kThreads, smem, st>>>((const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v, meta, sc.o,
+  launch_pdl(tree_attn_mma_kernel<DH>, dim3(grid), dim3(kThreads), smem, st, (const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v, meta, sc.o,
                                                         sc.ml, rows, n_heads, max_ctx);
 }
 

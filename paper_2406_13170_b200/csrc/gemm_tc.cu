@@ -16,6 +16,7 @@
 #include <tuple>
 
 #include "amph.h"
+#include "amph_internal.cuh"
 #include "gemm_tc.cuh"
 
 namespace amph {
@@ -131,6 +132,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
+  pdl_launch_dependents();                          // the consumer kernel may get resident and wait
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
@@ -166,8 +168,18 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       const CUtensorMap* wmap = &maps.w[seg];
       asm volatile("prefetch.tensormap [%0];" ::"l"(wmap) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x) : "memory");
-      int issued = 0;
-      for (int i = 0; i < nkb; ++i) {
+      // Weights do not depend on the previous kernel: fill the ring with weight tiles first, then wait for
+      // the producer of the activations, then fetch the activation tiles of those stages.
+      const int npre = nkb < stages ? nkb : stages;
+      for (int i = 0; i < npre; ++i) {
+        mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
+        tma_load_2d(smem + (size_t)i * stage_bytes, wmap, (kb_lo + i) * kTileK, row0, &full_bar[i]);
+      }
+      pdl_wait();
+      for (int i = 0; i < npre; ++i)
+        tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, (kb_lo + i) * kTileK, 0, &full_bar[i]);
+      int issued = npre;
+      for (int i = npre; i < nkb; ++i) {
         const int s = i % stages, round = i / stages;
         if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag)) break;
         uint8_t* a = smem + (size_t)s * stage_bytes;
@@ -207,6 +219,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   } else {
     // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
     const int quarter = warp & 3;
+    pdl_wait();                                      // P may still be read by the kernel before this one
     const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag) : false);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int feat = seg * prm.tiles_per_seg * kTileM + row0 + quarter * 32 + lane;
@@ -341,7 +354,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.stages = stages;
   prm.err_flag = g->err_flag;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  tc_gemm_kernel<<<dim3(tiles, splits), kThreads, smem, st>>>(pack, prm);
+  launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
   *split_stride = prm.split_stride;
   return true;

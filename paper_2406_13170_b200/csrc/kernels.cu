@@ -71,6 +71,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ emb, const int* __restrict__ toks, int vocab, int d,
                              float* __restrict__ x) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = blockIdx.x;
   int t = toks[r];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
@@ -80,7 +82,7 @@ __global__ void embed_kernel(const T* __restrict__ emb, const int* __restrict__ 
 
 void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d, float* x,
                   cudaStream_t st) {
-  AMPH_DISPATCH(dtype, embed_kernel<T><<<rows, 256, 0, st>>>((const T*)tok_emb, toks, vocab, d, x));
+  AMPH_DISPATCH(dtype, launch_pdl(embed_kernel<T>, dim3(rows), dim3(256), 0, st, (const T*)tok_emb, toks, vocab, d, x));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -90,6 +92,8 @@ template <typename T>
 __global__ void __launch_bounds__(1024)
 resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, const T* __restrict__ gain,
                   T* __restrict__ xn, float* __restrict__ hid, float eps, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ __align__(16) float rowbuf[];
   __shared__ float red[32];
   const int r = blockIdx.x;
@@ -130,7 +134,7 @@ void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const voi
                        void* xn, float* hid, float eps, int rows, int d, cudaStream_t st) {
   int threads = (d / 4 + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
-  AMPH_DISPATCH(dtype, resid_norm_kernel<T><<<rows, threads, d * sizeof(float), st>>>(
+  AMPH_DISPATCH(dtype, launch_pdl(resid_norm_kernel<T>, dim3(rows), dim3(threads), d * sizeof(float), st, 
                            x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d));
 }
 
@@ -139,6 +143,8 @@ void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const voi
 // --------------------------------------------------------------------------------------------
 __global__ void rope_table_kernel(const RowMeta* __restrict__ meta, const double* __restrict__ inv_freq,
                                   float2* __restrict__ table, int half) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = blockIdx.x;
   const double p = (double)meta->pos[r];
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
@@ -150,7 +156,7 @@ __global__ void rope_table_kernel(const RowMeta* __restrict__ meta, const double
 
 void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
                        cudaStream_t st) {
-  rope_table_kernel<<<rows, 64, 0, st>>>(meta, inv_freq, table, half);
+  launch_pdl(rope_table_kernel, dim3(rows), dim3(64), 0, st, meta, inv_freq, table, half);
 }
 
 // --------------------------------------------------------------------------------------------
@@ -160,6 +166,8 @@ template <typename T>
 __global__ void __launch_bounds__(1024)
 qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* __restrict__ rope, T* __restrict__ q,
                 T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = blockIdx.x;
   const int half = dh >> 1, d = n_heads * dh, quads = half >> 2;
   const bool live = r < meta->n_rows;
@@ -194,7 +202,7 @@ void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, voi
                      int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st) {
   int threads = (n_heads * head_dim / 8 + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
-  AMPH_DISPATCH(dtype, qkv_rope_kernel<T><<<rows, threads, 0, st>>>(P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
+  AMPH_DISPATCH(dtype, launch_pdl(qkv_rope_kernel<T>, dim3(rows), dim3(threads), 0, st, P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
                                                                     n_heads, head_dim, max_ctx));
 }
 
@@ -212,6 +220,8 @@ __global__ void __launch_bounds__(kAttThreads)
 tree_attn_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
                  const RowMeta* __restrict__ meta, float* __restrict__ po, float* __restrict__ pml,
                  int rows_cap, int n_heads, int max_ctx) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int QS = DH + 4;                       // padded row strides (bank-conflict free float4 reads)
   constexpr int SEG = DH / 4;                      // output dims owned by one thread
   extern __shared__ __align__(16) float sm[];
@@ -334,6 +344,8 @@ tree_attn_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __r
 template <typename T>
 __global__ void attn_combine_kernel(const float* __restrict__ po, const float* __restrict__ pml,
                                     T* __restrict__ out, int splits, int rows_cap, int n_heads, int dh) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = blockIdx.x, h = blockIdx.y;
   float M = -INFINITY;
   for (int s = 0; s < splits; ++s)
@@ -362,9 +374,9 @@ static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, Attn
                                        kAttRows * (kAttTile + 1));
   cudaFuncSetAttribute(tree_attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid(n_heads, splits, (rows + kAttRows - 1) / kAttRows);
-  tree_attn_kernel<T, DH><<<grid, kAttThreads, smem, st>>>((const T*)q, (const T*)kv.k, (const T*)kv.v, meta,
+  launch_pdl(tree_attn_kernel<T, DH>, dim3(grid), dim3(kAttThreads), smem, st, (const T*)q, (const T*)kv.k, (const T*)kv.v, meta,
                                                           sc.o, sc.ml, rows, n_heads, max_ctx);
-  attn_combine_kernel<T><<<dim3(rows, n_heads), DH < 128 ? 64 : 128, 0, st>>>(sc.o, sc.ml, (T*)out, splits, rows,
+  launch_pdl(attn_combine_kernel<T>, dim3(dim3(rows, n_heads)), dim3(DH < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (T*)out, splits, rows,
                                                                               n_heads, DH);
 }
 
@@ -376,7 +388,7 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
   if (splits < 1) splits = 1;
   if (dtype == AMPH_DTYPE_BF16) {                    // tensor-core path; the kernel below serves fp32 caches
     launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st);
-    attn_combine_kernel<bf16><<<dim3(rows, n_heads), head_dim < 128 ? 64 : 128, 0, st>>>(sc.o, sc.ml, (bf16*)out, splits,
+    launch_pdl(attn_combine_kernel<bf16>, dim3(dim3(rows, n_heads)), dim3(head_dim < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (bf16*)out, splits,
                                                                                         rows, n_heads, head_dim);
     return;
   }
@@ -392,6 +404,8 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 // --------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f) {
+  pdl_wait();
+  pdl_launch_dependents();
   const size_t n = (size_t)rows * f;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(i / f), c = (int)(i - (size_t)r * f);
@@ -404,7 +418,7 @@ void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStr
   const size_t n = (size_t)rows * f;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  AMPH_DISPATCH(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(P, (T*)act, rows, f));
+  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, P, (T*)act, rows, f));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -413,6 +427,8 @@ void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStr
 template <typename T>
 __global__ void concat_kernel(const float* __restrict__ feat, const T* __restrict__ emb,
                               const int* __restrict__ next_tok, int vocab, T* __restrict__ cat, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = blockIdx.x;
   int t = next_tok[r];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
@@ -424,7 +440,7 @@ __global__ void concat_kernel(const float* __restrict__ feat, const T* __restric
 
 void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat, int dtype,
                    int rows, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, concat_kernel<T><<<rows, 256, 0, st>>>(feat, (const T*)tok_emb, next_tok, vocab, (T*)cat, d));
+  AMPH_DISPATCH(dtype, launch_pdl(concat_kernel<T>, dim3(rows), dim3(256), 0, st, feat, (const T*)tok_emb, next_tok, vocab, (T*)cat, d));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -457,6 +473,8 @@ template <typename T, int R>
 __global__ void __launch_bounds__(256)
 gemm_generic_kernel(const T* __restrict__ X, int ldx, const T* __restrict__ W, int out, int in,
                     float* __restrict__ P, int ldp, int col_off, int rows) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int V = Vec16<T>::N;
   const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -492,7 +510,7 @@ void launch_gemm_generic(const void* x, int ldx, const GemmSeg* segs, int n_seg,
                          int ldp, int rows, int dtype, cudaStream_t st) {
   const int blocks = (out + 7) / 8;
   for (int s = 0; s < n_seg; ++s) {
-    AMPH_DISPATCH(dtype, gemm_generic_kernel<T, 8><<<blocks, 256, 0, st>>>(
+    AMPH_DISPATCH(dtype, launch_pdl(gemm_generic_kernel<T, 8>, dim3(blocks), dim3(256), 0, st, 
                              (const T*)x, ldx, (const T*)segs[s].w, out, in, P, ldp, s * out, rows));
   }
 }
@@ -504,6 +522,8 @@ template <typename T>
 __global__ void gather_last_kernel(const float* __restrict__ h1, const float* __restrict__ h2,
                                    const DevState* __restrict__ s, float* __restrict__ last,
                                    T* __restrict__ last_act, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   int lr = s->n_pending - 1;
   lr = lr < 0 ? 0 : (lr >= kPendMax ? kPendMax - 1 : lr);
   const float* src = blockIdx.x == 0 ? h1 : h2;
@@ -516,7 +536,7 @@ __global__ void gather_last_kernel(const float* __restrict__ h1, const float* __
 
 void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev, float* last, void* last_act,
                         int dtype, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, gather_last_kernel<T><<<2, 256, 0, st>>>(h1, h2, st_dev, last, (T*)last_act, d));
+  AMPH_DISPATCH(dtype, launch_pdl(gather_last_kernel<T>, dim3(2), dim3(256), 0, st, h1, h2, st_dev, last, (T*)last_act, d));
 }
 
 struct BiasPtrs { const void* b[kMaxK]; };
@@ -525,6 +545,8 @@ template <typename T>
 __global__ void mlp_heads_kernel(PartialView P, const float* __restrict__ last, BiasPtrs bias,
                                  const T* __restrict__ pe, float* __restrict__ hp, float* __restrict__ ao,
                                  T* __restrict__ ao_act, int K, int n_sal, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int k = blockIdx.x;
   const int row = (k < K / 2 || n_sal == 1) ? 0 : 1;       // Eq. 2: first half of the heads <- stage 1
   const T* b = (const T*)bias.b[k];
@@ -541,13 +563,15 @@ void launch_mlp_heads(PartialView P, const float* last, const void* const* bias,
                       float* ao, void* ao_act, int dtype, int K, int n_sal, int d, cudaStream_t st) {
   BiasPtrs bp;
   for (int k = 0; k < kMaxK; ++k) bp.b[k] = k < K ? bias[k] : nullptr;
-  AMPH_DISPATCH(dtype, mlp_heads_kernel<T><<<K, 256, 0, st>>>(P, last, bp, (const T*)pe, hp, ao, (T*)ao_act,
+  AMPH_DISPATCH(dtype, launch_pdl(mlp_heads_kernel<T>, dim3(K), dim3(256), 0, st, P, last, bp, (const T*)pe, hp, ao, (T*)ao_act,
                                                               K, n_sal, d));
 }
 
 // One block per attention head: the K x K score matrix, softmax and mixing stay in shared memory.
 template <typename T>
 __global__ void aeb_attention_kernel(PartialView P, T* __restrict__ out, int K, int n_heads, int dh) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ float sm[];
   float* qs = sm;                 // [K][dh]
   float* ks = qs + K * dh;
@@ -590,7 +614,7 @@ __global__ void aeb_attention_kernel(PartialView P, T* __restrict__ out, int K, 
 void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
                           cudaStream_t st) {
   const size_t smem = sizeof(float) * (3 * K * head_dim + K * K);
-  AMPH_DISPATCH(dtype, aeb_attention_kernel<T><<<n_heads, 128, smem, st>>>(P, (T*)out_act, K, n_heads, head_dim));
+  AMPH_DISPATCH(dtype, launch_pdl(aeb_attention_kernel<T>, dim3(n_heads), dim3(128), smem, st, P, (T*)out_act, K, n_heads, head_dim));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -620,6 +644,8 @@ struct TopkCounts { int c[kMaxK]; };
 
 __global__ void topk_heads_kernel(PartialView P, int vocab, TopkCounts ck, int* __restrict__ ids,
                                   float* __restrict__ vals, float* __restrict__ d_logits) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float sv[32];
   __shared__ int si[32];
   const int k = blockIdx.x;
@@ -647,11 +673,13 @@ void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids,
                        cudaStream_t st) {
   TopkCounts c;
   for (int k = 0; k < kMaxK; ++k) c.c[k] = k < K ? ck[k] : 0;
-  topk_heads_kernel<<<K, 1024, 0, st>>>(P, vocab, c, ids, vals, d_logits);
+  launch_pdl(topk_heads_kernel, dim3(K), dim3(1024), 0, st, P, vocab, c, ids, vals, d_logits);
 }
 
 __global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ amax,
                                    float* __restrict__ logits_out) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float sv[32];
   __shared__ int si[32];
   const int r = blockIdx.x;
@@ -667,7 +695,7 @@ __global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ a
 }
 
 void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st) {
-  argmax_rows_kernel<<<rows, 1024, 0, st>>>(P, vocab, amax, logits_out);
+  launch_pdl(argmax_rows_kernel, dim3(rows), dim3(1024), 0, st, P, vocab, amax, logits_out);
 }
 
 // --------------------------------------------------------------------------------------------
@@ -679,6 +707,8 @@ __device__ __forceinline__ void chain_mask(int r, u64* m) {       // bits 0..r
 }
 
 __global__ void meta_chain_kernel(RowMeta* meta, int base, int n_rows) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = threadIdx.x;
   if (r == 0) { meta->base = base; meta->n_rows = n_rows; }
   meta->pos[r] = base + r;
@@ -687,10 +717,12 @@ __global__ void meta_chain_kernel(RowMeta* meta, int base, int n_rows) {
 }
 
 void launch_meta_chain(RowMeta* meta, int base, int n_rows, cudaStream_t st) {
-  meta_chain_kernel<<<1, kMaxRows, 0, st>>>(meta, base, n_rows);
+  launch_pdl(meta_chain_kernel, dim3(1), dim3(kMaxRows), 0, st, meta, base, n_rows);
 }
 
 __global__ void meta_pending_kernel(RowMeta* meta, const DevState* s) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int r = threadIdx.x;
   int np = s->n_pending;
   np = np < 0 ? 0 : (np > kPendMax ? kPendMax : np);
@@ -702,13 +734,15 @@ __global__ void meta_pending_kernel(RowMeta* meta, const DevState* s) {
 }
 
 void launch_meta_pending(RowMeta* meta, const DevState* s, cudaStream_t st) {
-  meta_pending_kernel<<<1, kMaxRows, 0, st>>>(meta, s);
+  launch_pdl(meta_pending_kernel, dim3(1), dim3(kMaxRows), 0, st, meta, s);
 }
 
 // tok[0] = root; tok[n] = head depth[n]'s candidate of rank rank[n] (Appendix A.1); optional overrides;
 // row table of the verification pass: position C + depth, slot C + n, mask = ancestors (Fig. 5).
 __global__ void tree_build_kernel(const TreeDev* __restrict__ tree, DevState* s, const int* __restrict__ topk_ids,
                                   const int* __restrict__ override_tok, int* __restrict__ tok, RowMeta* meta) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int n = threadIdx.x;
   const int N = tree->n_nodes;
   const int C = s->C;
@@ -733,7 +767,7 @@ __global__ void tree_build_kernel(const TreeDev* __restrict__ tree, DevState* s,
 
 void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, const int* override_tok, int* tok,
                        RowMeta* meta, cudaStream_t st) {
-  tree_build_kernel<<<1, kMaxRows, 0, st>>>(tree, s, topk_ids, override_tok, tok, meta);
+  launch_pdl(tree_build_kernel, dim3(1), dim3(kMaxRows), 0, st, tree, s, topk_ids, override_tok, tok, meta);
 }
 
 // Greedy acceptance: node n matches if its token equals the target's choice at its parent; it is
@@ -741,6 +775,8 @@ void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, co
 // among equals).  One block; the match set is a 128-bit mask tested against the ancestor masks.
 __global__ void accept_kernel(const TreeDev* __restrict__ tree, DevState* s, const int* __restrict__ tok,
                               const int* __restrict__ amax) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ u64 match[2];
   __shared__ int best_key;
   const int n = threadIdx.x;
@@ -782,7 +818,7 @@ __global__ void accept_kernel(const TreeDev* __restrict__ tree, DevState* s, con
 }
 
 void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st) {
-  accept_kernel<<<1, kMaxRows, 0, st>>>(tree, s, tok, amax);
+  launch_pdl(accept_kernel, dim3(1), dim3(kMaxRows), 0, st, tree, s, tok, amax);
 }
 
 // Block l < n_layers moves layer l's accepted key / value rows: slot C_old + j <- C_old + path[j].
@@ -792,6 +828,8 @@ template <typename T>
 __global__ void compact_kernel(const DevState* __restrict__ s, const KvView* __restrict__ kv, int n_layers,
                                int n_heads, int dh, int max_ctx, const float* __restrict__ hidden,
                                float* __restrict__ pend_h, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int L = s->L, C0 = s->C_old;
   if ((int)blockIdx.x == n_layers) {
     for (int j = 0; j < L; ++j)
@@ -814,11 +852,13 @@ __global__ void compact_kernel(const DevState* __restrict__ s, const KvView* __r
 
 void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
                     int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, compact_kernel<T><<<n_layers + 1, 256, 0, st>>>(s, kv_layers, n_layers, n_heads, head_dim,
+  AMPH_DISPATCH(dtype, launch_pdl(compact_kernel<T>, dim3(n_layers + 1), dim3(256), 0, st, s, kv_layers, n_layers, n_heads, head_dim,
                                                                        max_ctx, hidden, pend_h, d));
 }
 
 __global__ void reduce_partials_kernel(PartialView P, float* __restrict__ y, int rows, int cols) {
+  pdl_wait();
+  pdl_launch_dependents();
   const size_t n = (size_t)rows * cols;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(i / cols), c = (int)(i - (size_t)r * cols);
@@ -830,12 +870,14 @@ void launch_reduce_partials(PartialView P, float* y, int rows, int cols, cudaStr
   const size_t n = (size_t)rows * cols;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  reduce_partials_kernel<<<blocks, 256, 0, st>>>(P, y, rows, cols);
+  launch_pdl(reduce_partials_kernel, dim3(blocks), dim3(256), 0, st, P, y, rows, cols);
 }
 
 template <typename T>
 __global__ void kv_export_kernel(const T* __restrict__ c, int row0, int n_heads, int dh, int max_ctx,
                                  float* __restrict__ dst) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int slot = row0 + blockIdx.x;
   for (int i = threadIdx.x; i < n_heads * dh; i += blockDim.x) {
     const int h = i / dh, e = i - h * dh;
@@ -846,7 +888,7 @@ __global__ void kv_export_kernel(const T* __restrict__ c, int row0, int n_heads,
 void launch_kv_export(KvView kv, int which, int dtype, int row0, int rows, int n_heads, int head_dim, int max_ctx,
                       float* dst, cudaStream_t st) {
   if (rows <= 0) return;
-  AMPH_DISPATCH(dtype, kv_export_kernel<T><<<rows, 256, 0, st>>>((const T*)(which ? kv.v : kv.k), row0, n_heads,
+  AMPH_DISPATCH(dtype, launch_pdl(kv_export_kernel<T>, dim3(rows), dim3(256), 0, st, (const T*)(which ? kv.v : kv.k), row0, n_heads,
                                                                  head_dim, max_ctx, dst));
 }
 
@@ -854,6 +896,8 @@ void launch_kv_export(KvView kv, int which, int dtype, int row0, int rows, int n
 // pending so that the first draft runs the adaptation layers on it (Eq. 1).
 __global__ void prefill_tail_kernel(DevState* s, const int* __restrict__ amax, int last_row,
                                     const float* __restrict__ hidden, float* __restrict__ pend_h, int d, int C) {
+  pdl_wait();
+  pdl_launch_dependents();
   for (int c = threadIdx.x; c < d; c += blockDim.x) pend_h[c] = hidden[(size_t)last_row * d + c];
   if (threadIdx.x == 0) {
     const int root = amax[last_row];
@@ -870,7 +914,7 @@ __global__ void prefill_tail_kernel(DevState* s, const int* __restrict__ amax, i
 
 void launch_prefill_tail(DevState* s, const int* amax, int last_row, const float* hidden, float* pend_h, int d,
                          int C, cudaStream_t st) {
-  prefill_tail_kernel<<<1, 256, 0, st>>>(s, amax, last_row, hidden, pend_h, d, C);
+  launch_pdl(prefill_tail_kernel, dim3(1), dim3(256), 0, st, s, amax, last_row, hidden, pend_h, d, C);
 }
 
 }  // namespace amph
