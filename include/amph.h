@@ -188,6 +188,17 @@ amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32
  * the bracketed launches: device time in milliseconds, number of launches, and weight bytes streamed
  * (each weight matrix counted once per launch).  HOST output pointers, each may be NULL.  At most
  * 16384 launches are recorded per begin / end pair; later ones run unrecorded. */
+enum {
+  AMPH_PROF_PROJECTION = 0,  /* weight-streaming projections                          */
+  AMPH_PROF_NORM = 1,        /* split-K reduction + residual + RMSNorm               */
+  AMPH_PROF_ROPE_KV = 2,     /* rotary embedding + KV-cache write                     */
+  AMPH_PROF_ATTENTION = 3,   /* tree attention (+ merge of the KV splits), Eq. 5 attention */
+  AMPH_PROF_SWIGLU = 4,
+  AMPH_PROF_SELECT = 5,      /* top-k per drafting head, argmax per verified row       */
+  AMPH_PROF_ACCEPT = 6,      /* acceptance + KV compaction                            */
+  AMPH_PROF_OTHER = 7,       /* embedding, concatenation, row tables, head epilogues   */
+  AMPH_PROF_CATEGORIES = 8
+};
 amph_status amph_profile_begin(amph_ctx* ctx);
 amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launches, int64_t* proj_weight_bytes);
 
@@ -227,6 +238,11 @@ amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* cons
 amph_status amph_project_noalloc(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
                                  int32_t out, int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core,
                                  float* y_dev, int32_t* status_dev, void* stream, char* err_msg, size_t err_len);
+
+/* Per-category device time of the last amph_profile_begin / amph_profile_end pair: ms and launches are
+ * HOST arrays of AMPH_PROF_CATEGORIES entries (either may be NULL).  While profiling, every kernel launch
+ * (or pair: attention + merge) is bracketed by events, which serialises kernels that otherwise overlap. */
+amph_status amph_profile_breakdown(amph_ctx* ctx, double* ms, int64_t* launches);
 
 /* Forgets the sequence (caches are logically emptied); weights stay registered. */
 amph_status amph_reset(amph_ctx* ctx);

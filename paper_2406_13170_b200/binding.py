@@ -23,7 +23,7 @@ STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
 EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
-           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_project", "amph_project_noalloc",
+           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_profile_breakdown", "amph_project", "amph_project_noalloc",
            "amph_reset", "amph_destroy", "amph_last_error"]
 
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         L.amph_get_state.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.amph_profile_begin.argtypes = [vp]
         L.amph_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.amph_profile_breakdown.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.amph_project.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_int32, vp, vp, C.c_size_t, vp]
         L.amph_project_noalloc.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -244,6 +245,14 @@ class Amphista:
         with torch.cuda.device(self.device):
             self._check(self.L.amph_profile_end(self.ctx, C.byref(ms), C.byref(n), C.byref(by)), self.ctx)
         return ms.value, n.value, by.value
+
+    PROF_NAMES = ["projection", "norm", "rope_kv", "attention", "swiglu", "select", "accept", "other"]
+
+    def profile_breakdown(self):
+        ms = (C.c_double * 8)()
+        n = (C.c_int64 * 8)()
+        self._check(self.L.amph_profile_breakdown(self.ctx, ms, n), self.ctx)
+        return {k: (ms[i], n[i]) for i, k in enumerate(self.PROF_NAMES)}
 
     def reset(self) -> None:
         self._check(self.L.amph_reset(self.ctx), self.ctx)

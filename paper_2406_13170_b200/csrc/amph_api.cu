@@ -80,8 +80,11 @@ struct amph_ctx {
   bool graph_off = false;   // capture is not possible (legacy stream, flag) or failed once
   bool prof_on = false;     // bracket projection launches with events (amph_profile_begin / end)
   std::vector<cudaEvent_t> prof_ev;
+  std::vector<int> prof_cat;
   size_t prof_used = 0;
   int64_t prof_bytes = 0;
+  double prof_cat_ms[AMPH_PROF_CATEGORIES] = {0};
+  int64_t prof_cat_n[AMPH_PROF_CATEGORIES] = {0};
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -98,6 +101,25 @@ amph_status fail(amph_ctx* ctx, amph_status code, const char* fmt, ...) {
   g_last_error = buf;
   return code;
 }
+
+// Brackets the launches issued during its lifetime with a pair of events (only while profiling).
+struct ProfScope {
+  amph_ctx* ctx;
+  bool rec;
+  ProfScope(amph_ctx* c, int cat) : ctx(c) {
+    rec = c->prof_on && c->prof_used + 2 <= c->prof_ev.size();
+    if (rec) {
+      cudaEventRecord(c->prof_ev[c->prof_used], c->stream);
+      c->prof_cat[c->prof_used / 2] = cat;
+    }
+  }
+  ~ProfScope() {
+    if (rec) {
+      cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], ctx->stream);
+      ctx->prof_used += 2;
+    }
+  }
+};
 
 amph_status cuda_check(amph_ctx* ctx, cudaError_t e, const char* what) {
   if (e == cudaSuccess) return AMPH_OK;
@@ -284,15 +306,9 @@ void* xbuf_ptr(amph_ctx* ctx, int xb) {
 PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows);
 
 PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
-  const bool rec = ctx->prof_on && ctx->prof_used + 2 <= ctx->prof_ev.size();
-  if (rec) cudaEventRecord(ctx->prof_ev[ctx->prof_used], ctx->stream);
-  PartialView pv = project_impl(ctx, xb, w, n_seg, out, in, rows);
-  if (rec) {
-    cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], ctx->stream);
-    ctx->prof_used += 2;
-    ctx->prof_bytes += (int64_t)n_seg * out * in * (int64_t)ctx->esz;
-  }
-  return pv;
+  ProfScope ps(ctx, AMPH_PROF_PROJECTION);
+  if (ps.rec) ctx->prof_bytes += (int64_t)n_seg * out * in * (int64_t)ctx->esz;
+  return project_impl(ctx, xb, w, n_seg, out, in, rows);
 }
 
 PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
@@ -329,20 +345,30 @@ void layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   cudaStream_t st = ctx->stream;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
   PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
   launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st);
+  }
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
+  { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
   launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
                         c.max_ctx, ctx_hi, l.attn_splits, st);
+  }
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_NORM);
   launch_resid_norm(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows, c.d_model, st);
+  }
   const void* gu[2] = {w.w_gate, w.w_up};
   P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
   launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st);
+  }
   const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
+  { ProfScope ps(ctx, AMPH_PROF_NORM);
   launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, next_gain ? ctx->ws + l.xn : nullptr, hid, c.rms_eps, rows,
                     c.d_model, st);
+  }
 }
 
 // Target forward of the rows in `tok` under meta_v; leaves post-final-norm rows in hidden and xn.
@@ -353,11 +379,17 @@ void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
   const RowMeta* meta = ctx->at<RowMeta>(l.meta_v);
   float2* rope = ctx->at<float2>(l.rope_v);
   float* x = ctx->at<float>(l.x);
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
+  }
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_embed(ctx->tok_emb, ctx->dtype, ctx->at<int>(l.tok), c.vocab, rows, c.d_model, x, st);
+  }
   PartialView none = {nullptr, 0, 0, 0};
+  { ProfScope ps(ctx, AMPH_PROF_NORM);
   launch_resid_norm(x, none, 0, 0, ctx->layers[0].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                     c.d_model, st);
+  }
   for (int i = 0; i < c.n_layers; ++i) {
     const bool last = i + 1 == c.n_layers;
     layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
@@ -370,7 +402,9 @@ void target_head(amph_ctx* ctx, int rows) {
   const Layout& l = ctx->lay;
   const void* w[1] = {ctx->lm_head};
   PartialView P = project(ctx, XB_XN, w, 1, c.vocab, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_SELECT);
   launch_argmax_rows(P, c.vocab, rows, ctx->at<int>(l.amax), ctx->at<float>(l.logits), ctx->stream);
+  }
 }
 
 // Eq. 1: both adaptation stages over the rows (feat, next_tok) described by meta_s.
@@ -380,15 +414,21 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
   cudaStream_t st = ctx->stream;
   const RowMeta* meta = ctx->at<RowMeta>(l.meta_s);
   float2* rope = ctx->at<float2>(l.rope_s);
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
+  }
   const float* in_feat = feat;
   for (int s = 0; s < c.n_sal; ++s) {
     float* hbuf = ctx->at<float>(s == 0 ? l.h1 : l.h2);
+    { ProfScope ps(ctx, AMPH_PROF_OTHER);
     launch_concat(in_feat, ctx->tok_emb, next_tok, c.vocab, ctx->ws + l.cat, ctx->dtype, rows, c.d_model, st);
+    }
     const void* w[1] = {ctx->fc[s]};
     PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, 2 * c.d_model, rows);
+    { ProfScope ps(ctx, AMPH_PROF_NORM);
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
+    }
     layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr);
     in_feat = hbuf;
   }
@@ -417,26 +457,40 @@ amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
   cudaStream_t st = ctx->stream;
   DevState* ds = ctx->at<DevState>(l.state);
   const int rows = ctx->rows_small;
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_meta_pending(ctx->at<RowMeta>(l.meta_s), ds, st);
+  }
   run_sals(ctx, ctx->at<float>(l.pend_h), ds->pend_tok, rows, ctx->ctx_hi);
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_gather_last(ctx->at<float>(l.h1), ctx->at<float>(c.n_sal == 2 ? l.h2 : l.h1), ds, ctx->at<float>(l.last),
                      ctx->ws + l.last_act, ctx->dtype, c.d_model, st);
+  }
   PartialView P = project(ctx, XB_LAST, ctx->mlp_w, c.K, c.d_model, c.d_model, 2);                   // Eq. 2
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_mlp_heads(P, ctx->at<float>(l.last), ctx->mlp_b, ctx->pe, ctx->at<float>(l.hp), ctx->at<float>(l.attn_o),
                    ctx->ws + l.ao_act, ctx->dtype, c.K, c.n_sal, c.d_model, st);                      // Eq. 3-4
+  }
   for (int a = 0; a < c.aeb_layers; ++a) {                                                            // Eq. 5
     P = project(ctx, XB_AO, ctx->aeb_w[a], 3, c.d_model, c.d_model, c.K);
+    { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
     launch_aeb_attention(P, ctx->ws + l.aeb_act, ctx->dtype, c.K, c.n_heads, c.head_dim, st);
+    }
     const void* wo[1] = {ctx->aeb_w[a][3]};
     P = project(ctx, XB_AEB, wo, 1, c.d_model, c.d_model, c.K);
+    { ProfScope ps(ctx, AMPH_PROF_NORM);
     launch_resid_norm(ctx->at<float>(l.attn_o), P, 0, 1, nullptr, ctx->dtype, ctx->ws + l.ao_act, nullptr, c.rms_eps,
                       c.K, c.d_model, st);
+    }
   }
   P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                               // Eq. 6
+  { ProfScope ps(ctx, AMPH_PROF_SELECT);
   launch_topk_heads(P, c.vocab, c.K, c.topk, ctx->at<int>(l.topk_ids), ctx->at<float>(l.topk_vals),
                     ctx->at<float>(l.d_logits), st);
+  }
+  { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_tree_build(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.topk_ids), nullptr, ctx->at<int>(l.tok),
                     ctx->at<RowMeta>(l.meta_v), st);
+  }
   amph_status rc = copy_out(ctx, out_ids, ctx->at<int>(l.topk_ids), sizeof(int) * c.K * kTopkStride);
   if (rc == AMPH_OK) rc = copy_out(ctx, out_vals, ctx->at<float>(l.topk_vals), sizeof(float) * c.K * kTopkStride);
   return rc;
@@ -450,8 +504,10 @@ amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_ar
     amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.override_tok), tree_tokens, sizeof(int) * N,
                                                      cudaMemcpyDefault, st), "copy of tree tokens");
     if (rc != AMPH_OK) return rc;
+    { ProfScope ps(ctx, AMPH_PROF_OTHER);
     launch_tree_build(ctx->at<TreeDev>(l.tree), ctx->at<DevState>(l.state), nullptr, ctx->at<int>(l.override_tok),
                       ctx->at<int>(l.tok), ctx->at<RowMeta>(l.meta_v), st);
+    }
   }
   target_forward(ctx, ctx->Mcap, ctx->ctx_hi + N);
   target_head(ctx, ctx->Mcap);
@@ -463,9 +519,13 @@ amph_status do_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
   DevState* ds = ctx->at<DevState>(l.state);
+  { ProfScope ps(ctx, AMPH_PROF_ACCEPT);
   launch_accept(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.tok), ctx->at<int>(l.amax), st);
+  }
+  { ProfScope ps(ctx, AMPH_PROF_ACCEPT);
   launch_compact(ds, ctx->at<KvView>(l.kv_tab), c.n_layers, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx,
                  ctx->at<float>(l.hidden), ctx->at<float>(l.pend_h), c.d_model, st);
+  }
   amph_status rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
   if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
   if (rc == AMPH_OK) rc = copy_out(ctx, out_path, ds->path, sizeof(int) * (c.K + 1));
@@ -797,6 +857,7 @@ amph_status amph_profile_begin(amph_ctx* ctx) {
         return cuda_check(ctx, cudaGetLastError(), "event creation");
       }
   }
+  ctx->prof_cat.assign(ctx->prof_ev.size() / 2, 0);
   ctx->prof_used = 0;
   ctx->prof_bytes = 0;
   ctx->prof_on = true;
@@ -809,13 +870,17 @@ amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launc
   ctx->prof_on = false;
   amph_status rc = cuda_check(ctx, cudaStreamSynchronize(ctx->stream), "profile synchronise");
   if (rc != AMPH_OK) return rc;
-  double ms = 0.0;
+  for (int c = 0; c < AMPH_PROF_CATEGORIES; ++c) { ctx->prof_cat_ms[c] = 0.0; ctx->prof_cat_n[c] = 0; }
   for (size_t i = 0; i + 1 < ctx->prof_used; i += 2) {
     float t = 0.f;
-    if (cudaEventElapsedTime(&t, ctx->prof_ev[i], ctx->prof_ev[i + 1]) == cudaSuccess) ms += t;
+    const int cat = ctx->prof_cat[i / 2];
+    if (cudaEventElapsedTime(&t, ctx->prof_ev[i], ctx->prof_ev[i + 1]) == cudaSuccess) {
+      ctx->prof_cat_ms[cat] += t;
+      ctx->prof_cat_n[cat] += 1;
+    }
   }
-  if (proj_ms) *proj_ms = ms;
-  if (proj_launches) *proj_launches = (int64_t)(ctx->prof_used / 2);
+  if (proj_ms) *proj_ms = ctx->prof_cat_ms[AMPH_PROF_PROJECTION];
+  if (proj_launches) *proj_launches = ctx->prof_cat_n[AMPH_PROF_PROJECTION];
   if (proj_weight_bytes) *proj_weight_bytes = ctx->prof_bytes;
   return AMPH_OK;
 }
@@ -861,6 +926,15 @@ amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* cons
   }
   launch_reduce_partials(pv, y_dev, rows, (int)ld, st);
   return cuda_check(nullptr, cudaGetLastError(), "projection");
+}
+
+amph_status amph_profile_breakdown(amph_ctx* ctx, double* ms, int64_t* launches) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  for (int c = 0; c < AMPH_PROF_CATEGORIES; ++c) {
+    if (ms) ms[c] = ctx->prof_cat_ms[c];
+    if (launches) launches[c] = ctx->prof_cat_n[c];
+  }
+  return AMPH_OK;
 }
 
 amph_status amph_reset(amph_ctx* ctx) {

@@ -45,6 +45,7 @@ struct TcParams {
   int nt;                   // activation rows in the MMA (multiple of 16)
   int rows;                 // live rows (only these are stored)
   int stages;
+  int l2_prefetch;          // weight tiles (beyond the ring) each CTA pulls into L2 before it waits
   int* err_flag;
 };
 
@@ -86,6 +87,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
   *abort_flag = 1;
   return false;
+}
+
+// Asks the TMA unit to bring one weight tile into L2 (no shared-memory destination, no barrier).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -175,6 +181,9 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
         tma_load_2d(smem + (size_t)i * stage_bytes, wmap, (kb_lo + i) * kTileK, row0, &full_bar[i]);
       }
+      // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
+      const int npf = nkb < npre + prm.l2_prefetch ? nkb : npre + prm.l2_prefetch;
+      for (int i = npre; i < npf; ++i) tma_prefetch_l2_2d(wmap, (kb_lo + i) * kTileK, row0);
       pdl_wait();
       for (int i = 0; i < npre; ++i)
         tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, (kb_lo + i) * kTileK, 0, &full_bar[i]);
@@ -352,6 +361,12 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.nt = nt;
   prm.rows = rows;
   prm.stages = stages;
+  // about 40 MB of L2 for prefetched weight tiles, shared by the CTAs that can be resident at once
+  {
+    const long long resident = (long long)tiles * splits < 2LL * g->sm_count ? (long long)tiles * splits : 2LL * g->sm_count;
+    long long pf = (40LL << 20) / (resident * (kTileM * kTileK * 2));
+    prm.l2_prefetch = (int)(pf > 32 ? 32 : pf);
+  }
   prm.err_flag = g->err_flag;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
