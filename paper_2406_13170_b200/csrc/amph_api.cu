@@ -336,55 +336,38 @@ PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg,
   return pv;
 }
 
-// Ranges of the next projection's weights for a kernel to pull into L2 (at most `cap` bytes in total).
-L2Prefetch prefetch_of(const amph_ctx* ctx, const void* const* w, int n, size_t elems_each, size_t cap = (size_t)48 << 20) {
-  L2Prefetch pf;
-  if (n < 1 || n > 3) return pf;
-  size_t each = elems_each * ctx->esz;
-  if (each * n > cap) each = (cap / n) & ~(size_t)127;
-  for (int i = 0; i < n; ++i) { pf.p[i] = w[i]; pf.bytes[i] = each; }
-  return pf;
-}
-
 // One decoder layer over the rows described by `meta`.  On entry xn holds RMSNorm(x) * attn_norm;
 // on exit x is updated and, if next_gain is given, xn (and hid) hold RMSNorm(x) * next_gain.
-// Each L2-resident kernel between two projections prefetches the head of the next projection's weights;
-// `after` names what follows this layer.
 void layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
-                   int rows, int ctx_hi, const void* next_gain, float* hid, L2Prefetch after) {
+                   int rows, int ctx_hi, const void* next_gain, float* hid) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const size_t dd = (size_t)c.d_model * c.d_model, df = (size_t)c.d_model * c.d_ffn;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
-  const void* wo[1] = {w.wo};
-  const void* wg[1] = {w.w_gate};
-  const void* wu[1] = {w.w_up};
-  const void* wd[1] = {w.w_down};
   PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
-  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st,
-                  prefetch_of(ctx, wo, 1, dd));
+  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st);
   }
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
   launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
-                        c.max_ctx, ctx_hi, l.attn_splits, st, prefetch_of(ctx, wg, 1, df));
+                        c.max_ctx, ctx_hi, l.attn_splits, st);
   }
+  const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_NORM);
-  launch_resid_norm(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows, c.d_model, st,
-                    prefetch_of(ctx, wu, 1, df));
+  launch_resid_norm(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows, c.d_model, st);
   }
   const void* gu[2] = {w.w_gate, w.w_up};
   P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
-  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, prefetch_of(ctx, wd, 1, df));
+  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st);
   }
+  const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
   { ProfScope ps(ctx, AMPH_PROF_NORM);
   launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, next_gain ? ctx->ws + l.xn : nullptr, hid, c.rms_eps, rows,
-                    c.d_model, st, after);
+                    c.d_model, st);
   }
 }
 
@@ -409,13 +392,8 @@ void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
   }
   for (int i = 0; i < c.n_layers; ++i) {
     const bool last = i + 1 == c.n_layers;
-    const void* nq[3] = {nullptr, nullptr, nullptr};
-    const void* nh[1] = {ctx->lm_head};
-    if (!last) { nq[0] = ctx->layers[i + 1].wq; nq[1] = ctx->layers[i + 1].wk; nq[2] = ctx->layers[i + 1].wv; }
     layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
-                  last ? ctx->final_norm : ctx->layers[i + 1].attn_norm, last ? ctx->at<float>(l.hidden) : nullptr,
-                  last ? prefetch_of(ctx, nh, 1, (size_t)c.vocab * c.d_model)
-                       : prefetch_of(ctx, nq, 3, (size_t)c.d_model * c.d_model));
+                  last ? ctx->final_norm : ctx->layers[i + 1].attn_norm, last ? ctx->at<float>(l.hidden) : nullptr);
   }
 }
 
@@ -451,9 +429,7 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
     }
-    const void* nfc[1] = {s + 1 < c.n_sal ? ctx->fc[s + 1] : ctx->mlp_w[0]};
-    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr,
-                  prefetch_of(ctx, nfc, 1, s + 1 < c.n_sal ? 2 * (size_t)c.d_model * c.d_model : (size_t)c.d_model * c.d_model));
+    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr);
     in_feat = hbuf;
   }
 }

@@ -78,33 +78,6 @@ inline cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_
 }
 #endif
 
-// Up to three address ranges (the next projection's weights) that a kernel asks the memory system to
-// pull into L2 while it does its own, L2-resident, work: HBM would otherwise idle between projections.
-struct L2Prefetch {
-  const void* p[3] = {nullptr, nullptr, nullptr};
-  unsigned long long bytes[3] = {0, 0, 0};
-};
-
-#ifdef __CUDACC__
-// Each CTA takes an equal slice of every range; one thread issues bulk L2 prefetches of <= 32 KB.
-__device__ __forceinline__ void l2_prefetch_slice(const L2Prefetch& pf) {
-  const unsigned long long nb = (unsigned long long)gridDim.x * gridDim.y * gridDim.z;
-  const unsigned long long b = blockIdx.x + (unsigned long long)gridDim.x * (blockIdx.y + (unsigned long long)gridDim.y * blockIdx.z);
-#pragma unroll
-  for (int i = 0; i < 3; ++i) {
-    if (pf.p[i] == nullptr || pf.bytes[i] == 0) continue;
-    const unsigned long long per = ((pf.bytes[i] + nb - 1) / nb + 127ull) & ~127ull;
-    unsigned long long lo = b * per;
-    const unsigned long long hi = lo + per < pf.bytes[i] ? lo + per : pf.bytes[i];
-    for (; lo < hi; lo += 32768ull) {
-      unsigned n = (unsigned)(hi - lo < 32768ull ? hi - lo : 32768ull);
-      n &= ~15u;
-      if (n) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((const char*)pf.p[i] + lo), "r"(n) : "memory");
-    }
-  }
-}
-#endif
-
 struct KvView {             // one layer's cache: K and V as [n_heads][max_ctx][head_dim]
   void* k;
   void* v;
@@ -126,15 +99,14 @@ void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, in
 // into xn (storage dtype) and hid (fp32); with gain == NULL xn / hid receive the plain row.
 // col_off selects the column window of P.
 void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
-                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st, L2Prefetch pf = L2Prefetch());
+                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st);
 
 void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
                        cudaStream_t st);
 
 // q <- rope(sum P[:, 0:d]); K cache <- rope(sum P[:, d:2d]); V cache <- sum P[:, 2d:3d]
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv,
-                     int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st,
-                     L2Prefetch pf = L2Prefetch());
+                     int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st);
 
 struct AttnScratch {
   float* o;                 // [splits][heads][rows][head_dim]
@@ -142,12 +114,12 @@ struct AttnScratch {
 };
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out,
                            int dtype, int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi,
-                           int max_splits, cudaStream_t st, L2Prefetch pf = L2Prefetch());
+                           int max_splits, cudaStream_t st);
 
 void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
-                               int head_dim, int max_ctx, int splits, cudaStream_t st, L2Prefetch pf);
+                               int head_dim, int max_ctx, int splits, cudaStream_t st);
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, L2Prefetch pf = L2Prefetch());
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st);
 
 // cat[r] = [feat[r] ; tok_emb[next[r]]]   (Eq. 1's concatenation)
 void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat,

@@ -67,10 +67,9 @@ template <int DH>
 __global__ void __launch_bounds__(kThreads)
 tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, const bf16* __restrict__ vc,
                      const RowMeta* __restrict__ meta, float* __restrict__ po, float* __restrict__ pml,
-                     int rows_cap, int n_heads, int max_ctx, L2Prefetch pf) {
+                     int rows_cap, int n_heads, int max_ctx) {
   pdl_wait();
   pdl_launch_dependents();
-  if (threadIdx.x == 0) l2_prefetch_slice(pf);
   constexpr int KS = DH / 16;                        // k-steps over the head dimension
   constexpr int NT = DH / 8;                         // 8-wide output tiles
   extern __shared__ __align__(128) unsigned char sm_raw[];
@@ -244,20 +243,20 @@ tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, co
 
 template <int DH>
 void launch_t(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads, int max_ctx,
-              int splits, cudaStream_t st, L2Prefetch pf) {
+              int splits, cudaStream_t st) {
   const size_t smem = sizeof(bf16) * (kRows * DH + 4 * kKeys * DH);
   cudaFuncSetAttribute(tree_attn_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid(n_heads, splits, (rows + kRows - 1) / kRows);
   launch_pdl(tree_attn_mma_kernel<DH>, dim3(grid), dim3(kThreads), smem, st, (const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v, meta, sc.o,
-                                                        sc.ml, rows, n_heads, max_ctx, pf);
+                                                        sc.ml, rows, n_heads, max_ctx);
 }
 
 }  // namespace
 
 void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
-                               int head_dim, int max_ctx, int splits, cudaStream_t st, L2Prefetch pf) {
-  if (head_dim == 64) launch_t<64>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st, pf);
-  else launch_t<128>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st, pf);
+                               int head_dim, int max_ctx, int splits, cudaStream_t st) {
+  if (head_dim == 64) launch_t<64>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st);
+  else launch_t<128>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st);
 }
 
 }  // namespace amph

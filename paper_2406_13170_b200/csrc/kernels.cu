@@ -91,10 +91,9 @@ void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, in
 template <typename T>
 __global__ void __launch_bounds__(1024)
 resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, const T* __restrict__ gain,
-                  T* __restrict__ xn, float* __restrict__ hid, float eps, int d, L2Prefetch pf) {
+                  T* __restrict__ xn, float* __restrict__ hid, float eps, int d) {
   pdl_wait();
   pdl_launch_dependents();
-  if (threadIdx.x == 0) l2_prefetch_slice(pf);
   extern __shared__ __align__(16) float rowbuf[];
   __shared__ float red[32];
   const int r = blockIdx.x;
@@ -132,11 +131,11 @@ resid_norm_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, c
 }
 
 void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
-                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st, L2Prefetch pf) {
+                       void* xn, float* hid, float eps, int rows, int d, cudaStream_t st) {
   int threads = (d / 4 + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
   AMPH_DISPATCH(dtype, launch_pdl(resid_norm_kernel<T>, dim3(rows), dim3(threads), d * sizeof(float), st, 
-                           x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d, pf));
+                           x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -166,10 +165,9 @@ void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* tabl
 template <typename T>
 __global__ void __launch_bounds__(1024)
 qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* __restrict__ rope, T* __restrict__ q,
-                T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx, L2Prefetch pf) {
+                T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
   pdl_wait();
   pdl_launch_dependents();
-  if (threadIdx.x == 0) l2_prefetch_slice(pf);
   const int r = blockIdx.x;
   const int half = dh >> 1, d = n_heads * dh, quads = half >> 2;
   const bool live = r < meta->n_rows;
@@ -201,11 +199,11 @@ qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* _
 }
 
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv, int dtype,
-                     int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st, L2Prefetch pf) {
+                     int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st) {
   int threads = (n_heads * head_dim / 8 + 31) / 32 * 32;
   if (threads > 1024) threads = 1024;
   AMPH_DISPATCH(dtype, launch_pdl(qkv_rope_kernel<T>, dim3(rows), dim3(threads), 0, st, P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
-                                                                    n_heads, head_dim, max_ctx, pf));
+                                                                    n_heads, head_dim, max_ctx));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -384,12 +382,12 @@ static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, Attn
 
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out, int dtype,
                            int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi, int max_splits,
-                           cudaStream_t st, L2Prefetch pf) {
+                           cudaStream_t st) {
   int splits = (ctx_hi + 127) / 128;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
   if (dtype == AMPH_DTYPE_BF16) {                    // tensor-core path; the kernel below serves fp32 caches
-    launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st, pf);
+    launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st);
     launch_pdl(attn_combine_kernel<bf16>, dim3(dim3(rows, n_heads)), dim3(head_dim < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (bf16*)out, splits,
                                                                                         rows, n_heads, head_dim);
     return;
@@ -405,10 +403,9 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 // SwiGLU on the fused gate / up projection: act = silu(gate) * up
 // --------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f, L2Prefetch pf) {
+__global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f) {
   pdl_wait();
   pdl_launch_dependents();
-  if (threadIdx.x == 0) l2_prefetch_slice(pf);
   const size_t n = (size_t)rows * f;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(i / f), c = (int)(i - (size_t)r * f);
@@ -417,11 +414,11 @@ __global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int 
   }
 }
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, L2Prefetch pf) {
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st) {
   const size_t n = (size_t)rows * f;
   int blocks = (int)((n + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, P, (T*)act, rows, f, pf));
+  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, P, (T*)act, rows, f));
 }
 
 // --------------------------------------------------------------------------------------------
