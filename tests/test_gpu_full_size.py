@@ -1,0 +1,57 @@
+"""Parity at the benchmark's full size and at the other large shapes.
+
+The 7B-shape test runs the exact configuration bench.py times (32 layers, d = 4096, vocab 32000, 64-node
+tree, 512-token prompt, tensor-core projections, CUDA-graph step) and compares it with the float32 CPU
+oracle on the same seeded weights: root token, draft logits and candidates, all 64 verified rows, acceptance
+and the compacted cache, for one natural and one planted step.  The 13B / 33B shapes are checked at two
+layers of depth (their widths, head counts and tile counts are what differs from 7B).
+"""
+import pytest
+import torch
+
+import inputs
+from oracle import amphista_oracle as ao
+from tests.parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TIE_BF16 = 1e-3
+
+
+def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1)):
+    from paper_2406_13170_b200 import Amphista
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
+    w_cpu = {k: v.cpu() for k, v in w_gpu.items()}                 # same generator; device independence is tested elsewhere
+    probe = inputs.normal_tensor(w_cpu["layers.0.wq"].shape, 0.02, 0, "layers.0.wq", dtype=torch.bfloat16)
+    assert torch.equal(probe, w_cpu["layers.0.wq"])
+    model = Amphista(shape, topo, w_gpu)
+    orc = ao.Oracle(shape, w_cpu, dtype=torch.float32)
+    prompt = inputs.make_prompt(shape, n=prompt_len or shape.prompt_len).tolist()
+    rep = run_parity(model, orc, shape, topo, prompt, steps, TOL_BF16, TIE_BF16, planted, kv_check_layers=kv_layers)
+    print(shape.name, rep)
+    # the same context must also run through amph_step (graph replay) and stay consistent with its own state
+    out_tok = torch.zeros(shape.K + 1, dtype=torch.int32, device="cuda:0")
+    out_n = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    C0 = model.get_state()[0]
+    for _ in range(3):
+        model.step(out_tok, out_n)
+    model.synchronize()
+    C1 = model.get_state()[0]
+    assert 3 <= C1 - C0 <= 3 * (shape.K + 1) and 1 <= int(out_n[0]) <= shape.K + 1
+    model.close()
+    return rep
+
+
+def test_7b_shape_full_depth():
+    shape = inputs.get_shape("7b")
+    rep = _run(shape, 2, True)
+    assert rep.steps == 2 and max(rep.accepted) >= 2
+
+
+@pytest.mark.parametrize("name", ["13b", "33b"])
+def test_large_shapes_two_layers(name):
+    shape = inputs.get_shape(name).with_(n_layers=2, prompt_len=70)
+    rep = _run(shape, 2, True, kv_layers=(0, 1))
+    assert rep.steps == 2
