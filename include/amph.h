@@ -174,7 +174,7 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
 
 /* Test hook: overwrites "tree_tokens" or "argmax" (i32 [n_nodes], host or device source) with a
  * stream-ordered copy, e.g. to run amph_accept on a chosen verification outcome.  Allowed after
- * amph_verify_tree only. */
+ * amph_verify_tree only.  "root" (i32 [1]) replaces the root token; allowed right after amph_prefill only. */
 amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes);
 
 /* Synchronises the stream and reports the committed length, the current root token and the

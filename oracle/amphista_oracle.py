@@ -181,6 +181,7 @@ class State:
     kv: List[LayerCache]                 # target, one per layer
     sal_kv: List[LayerCache]             # one per adaptation layer
     pending: List[Tuple[torch.Tensor, int, int]]   # (h_j, token id at j+1, j)
+    last_logits: Optional[torch.Tensor] = None     # target logits of the last prompt position (set by prefill)
 
 
 class Oracle:
@@ -247,7 +248,7 @@ class Oracle:
         hid, logits = self.target_rows(prompt, list(range(n)), list(range(n)), vis, kv)
         root = argmax_lowest(logits[n - 1])
         pending = [(hid[j], int(prompt[j + 1]) if j + 1 < n else root, j) for j in range(n)]
-        return State(n, root, kv, [LayerCache() for _ in range(self.s.n_sal)], pending)
+        return State(n, root, kv, [LayerCache() for _ in range(self.s.n_sal)], pending, logits[n - 1])
 
     def greedy_ar(self, prompt: Sequence[int], n_new: int) -> List[int]:
         """Plain greedy autoregressive decoding of the target: the definition the speculative

@@ -823,6 +823,13 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
 amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
   if (!name || !src) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and src must not be NULL");
+  if (strcmp(name, "root") == 0) {               // right after prefill: replaces the greedy root token
+    if (ctx->phase != PH_READY || bytes != sizeof(int)) return fail(ctx, AMPH_ERR_STATE, "'root' takes one int32 right after amph_prefill");
+    DevState* ds = ctx->at<DevState>(ctx->lay.state);
+    amph_status rc = cuda_check(ctx, cudaMemcpyAsync(&ds->root, src, sizeof(int), cudaMemcpyDefault, ctx->stream), "set_tensor");
+    if (rc == AMPH_OK) rc = cuda_check(ctx, cudaMemcpyAsync(&ds->pend_tok[0], src, sizeof(int), cudaMemcpyDefault, ctx->stream), "set_tensor");
+    return rc;
+  }
   if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_set_tensor must follow amph_verify_tree");
   size_t off;
   if (strcmp(name, "tree_tokens") == 0) off = ctx->lay.tok;
