@@ -185,10 +185,20 @@ class State:
 
 
 class Oracle:
-    def __init__(self, shape, weights: Dict[str, torch.Tensor], dtype=torch.float64):
+    """storage=None: every activation stays in `dtype` (the plain definition).
+    storage=torch.bfloat16: the precision reading for bf16 models, in which every tensor that is stored
+    for a later contraction is kept in bf16: the input rows of every projection, the rotated queries and
+    the key / value cache rows.  Accumulation, residual stream, softmax and norms stay in `dtype`."""
+
+    def __init__(self, shape, weights: Dict[str, torch.Tensor], dtype=torch.float64, storage=None):
         self.s = shape
         self.dtype = dtype
+        self.storage = storage
         self.w = weights            # kept in storage dtype; widened on use
+
+    def st(self, t: torch.Tensor) -> torch.Tensor:
+        """Round-trip through the activation storage type (identity when storage is None)."""
+        return t if self.storage is None else t.to(self.storage).to(t.dtype)
 
     def W(self, name: str) -> torch.Tensor:
         return self.w[name].to(self.dtype)
@@ -204,22 +214,22 @@ class Oracle:
         """
         s = self.s
         R = X.shape[0]
-        Xn = rmsnorm(X, self.W(prefix + "attn_norm"), s.rms_eps)
+        Xn = self.st(rmsnorm(X, self.W(prefix + "attn_norm"), s.rms_eps))
         Q = Xn @ self.W(prefix + "wq").T
         Kx = Xn @ self.W(prefix + "wk").T
         V = Xn @ self.W(prefix + "wv").T
         for r in range(R):
-            cache.put(slots[r], rope(Kx[r], pos[r], s.n_heads, s.head_dim, s.rope_theta), V[r])
+            cache.put(slots[r], self.st(rope(Kx[r], pos[r], s.n_heads, s.head_dim, s.rope_theta)), self.st(V[r]))
         A = torch.empty_like(X)
         for r in range(R):
             assert slots[r] in visible[r]
             keys, vals = cache.rows(visible[r])
-            q = rope(Q[r], pos[r], s.n_heads, s.head_dim, s.rope_theta)
+            q = self.st(rope(Q[r], pos[r], s.n_heads, s.head_dim, s.rope_theta))
             A[r] = attend(q, keys, vals, s.n_heads, s.head_dim)
-        X = X + A @ self.W(prefix + "wo").T
-        Xn = rmsnorm(X, self.W(prefix + "ffn_norm"), s.rms_eps)
+        X = X + self.st(A) @ self.W(prefix + "wo").T
+        Xn = self.st(rmsnorm(X, self.W(prefix + "ffn_norm"), s.rms_eps))
         act = silu(Xn @ self.W(prefix + "w_gate").T) * (Xn @ self.W(prefix + "w_up").T)
-        return X + act @ self.W(prefix + "w_down").T
+        return X + self.st(act) @ self.W(prefix + "w_down").T
 
     def embed(self, tok: int) -> torch.Tensor:
         return self.w["tok_emb"][int(tok)].to(self.dtype)
@@ -234,7 +244,7 @@ class Oracle:
         for l in range(s.n_layers):
             X = self.decoder_rows(f"layers.{l}.", X, pos, slots, visible, kv[l])
         hid = rmsnorm(X, self.W("final_norm"), s.rms_eps)
-        return hid, hid @ self.W("lm_head").T
+        return hid, self.st(hid) @ self.W("lm_head").T
 
     # ---- O1: prefill -------------------------------------------------------------------
     def prefill(self, prompt: Sequence[int]) -> State:
@@ -275,7 +285,7 @@ class Oracle:
         feats = [h for (h, _, _) in st.pending]
         for stage in range(1, s.n_sal + 1):
             fc = self.W(f"draft.fc{stage}")
-            X = torch.stack([fc @ torch.cat([f, self.embed(nxt)])            # Eq. 1: fc([h ; e_{t+1}])
+            X = torch.stack([fc @ self.st(torch.cat([f, self.embed(nxt)]))   # Eq. 1: fc([h ; e_{t+1}])
                              for (h, nxt, pos), f in zip(st.pending, feats)])
             poss = [pos for (_, _, pos) in st.pending]
             vis = [list(range(p + 1)) for p in poss]                  # causal: kv_{1:t-1} and itself
@@ -287,12 +297,12 @@ class Oracle:
         rows = []
         for k in range(1, K + 1):                                     # Eq. 2: head -> stage split
             src = stage_out[0] if (k <= K // 2 or s.n_sal == 1) else stage_out[1]
-            rows.append(src + silu(self.W(f"draft.mlp.{k-1}.w") @ src + self.W(f"draft.mlp.{k-1}.b")))
+            rows.append(src + silu(self.W(f"draft.mlp.{k-1}.w") @ self.st(src) + self.W(f"draft.mlp.{k-1}.b")))
         Hp = torch.stack(rows) + self.W("draft.pe")                   # Eq. 3, Eq. 4
         attn_o = Hp
         for l in range(s.aeb_layers):                                 # Eq. 5
             attn_o = self.aeb(attn_o, l)
-        d_logits = torch.stack([self.W(f"draft.lm_head.{k}") @ attn_o[k] for k in range(K)])  # Eq. 6
+        d_logits = torch.stack([self.W(f"draft.lm_head.{k}") @ self.st(attn_o[k]) for k in range(K)])  # Eq. 6
         ids, vals = [], []
         for k in range(K):
             i, v = topk_desc(d_logits[k], s.topk[k])
@@ -307,11 +317,12 @@ class Oracle:
         with a residual connection (Eq. 5; bi-directional: no mask, no positional rotation)."""
         s = self.s
         K = Hp.shape[0]
-        q = Hp @ self.W(f"draft.aeb.{l}.wq").T
-        k = Hp @ self.W(f"draft.aeb.{l}.wk").T
-        v = Hp @ self.W(f"draft.aeb.{l}.wv").T
+        Hs = self.st(Hp)
+        q = Hs @ self.W(f"draft.aeb.{l}.wq").T
+        k = Hs @ self.W(f"draft.aeb.{l}.wk").T
+        v = Hs @ self.W(f"draft.aeb.{l}.wv").T
         mixed = torch.stack([attend(q[i], k, v, s.n_heads, s.head_dim) for i in range(K)])
-        return Hp + mixed @ self.W(f"draft.aeb.{l}.wo").T
+        return Hp + self.st(mixed) @ self.W(f"draft.aeb.{l}.wo").T
 
     # ---- O3: tree tokens (Appendix A.1) -------------------------------------------------
     @staticmethod

@@ -17,9 +17,18 @@ pytestmark = pytest.mark.gpu
 
 TOL_BF16 = 2e-2
 TIE_BF16 = 1e-3
+TOL_STORAGE = 5e-3      # against the oracle that stores projection inputs and KV rows in bf16 like the kernels
 
 
-def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1)):
+def tol_plain(n_layers: int) -> float:
+    """Against the oracle that keeps every activation in float32.  The bf16 storage points (projection
+    inputs, rotated queries, KV rows) inject an error that accumulates like a random walk over the layers
+    of a random-init model: measured 1.1e-2 at 2 layers, 2.1e-2 at 8, 3.5e-2 at 16, 4.0e-2 at 32 (7B
+    widths), and reproduced on the CPU by the oracle's bf16-storage mode.  2e-2 holds up to 4 layers."""
+    return TOL_BF16 * max(1.0, (n_layers / 4.0) ** 0.5)
+
+
+def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1), storage=None):
     from paper_2406_13170_b200 import Amphista
     topo = inputs.make_tree(shape.n_nodes, shape.topk)
     w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
@@ -27,9 +36,10 @@ def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1)):
     probe = inputs.normal_tensor(w_cpu["layers.0.wq"].shape, 0.02, 0, "layers.0.wq", dtype=torch.bfloat16)
     assert torch.equal(probe, w_cpu["layers.0.wq"])
     model = Amphista(shape, topo, w_gpu)
-    orc = ao.Oracle(shape, w_cpu, dtype=torch.float32)
+    orc = ao.Oracle(shape, w_cpu, dtype=torch.float32, storage=storage)
+    tol = TOL_STORAGE if storage is not None else tol_plain(shape.n_layers)
     prompt = inputs.make_prompt(shape, n=prompt_len or shape.prompt_len).tolist()
-    rep = run_parity(model, orc, shape, topo, prompt, steps, TOL_BF16, TIE_BF16, planted, kv_check_layers=kv_layers)
+    rep = run_parity(model, orc, shape, topo, prompt, steps, tol, TIE_BF16, planted, kv_check_layers=kv_layers)
     print(shape.name, rep)
     # the same context must also run through amph_step (graph replay) and stay consistent with its own state
     out_tok = torch.zeros(shape.K + 1, dtype=torch.int32, device="cuda:0")
@@ -44,14 +54,16 @@ def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1)):
     return rep
 
 
-def test_7b_shape_full_depth():
+@pytest.mark.parametrize("storage", [None, torch.bfloat16], ids=["plain-oracle", "bf16-storage-oracle"])
+def test_7b_shape_full_depth(storage):
     shape = inputs.get_shape("7b")
-    rep = _run(shape, 2, True)
+    rep = _run(shape, 2, True, storage=storage)
     assert rep.steps == 2 and max(rep.accepted) >= 2
 
 
+@pytest.mark.parametrize("storage", [None, torch.bfloat16], ids=["plain-oracle", "bf16-storage-oracle"])
 @pytest.mark.parametrize("name", ["13b", "33b"])
-def test_large_shapes_two_layers(name):
+def test_large_shapes_two_layers(name, storage):
     shape = inputs.get_shape(name).with_(n_layers=2, prompt_len=70)
-    rep = _run(shape, 2, True, kv_layers=(0, 1))
+    rep = _run(shape, 2, True, kv_layers=(0, 1), storage=storage)
     assert rep.steps == 2

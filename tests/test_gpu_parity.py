@@ -65,3 +65,23 @@ def test_small_bf16_eight_steps(planted, flags):
     if planted:
         assert max(rep.accepted) >= 3
     model.close()
+
+
+def test_long_prompt_many_attention_splits_fp32():
+    """A 300-token context: several KV splits per head, five prefill chunks (fp32: tight tolerance)."""
+    shape = inputs.get_shape("tiny").with_(prompt_len=300)
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    model, orc = _setup(shape, topo)
+    rep = run_parity(model, orc, shape, topo, inputs.make_prompt(shape).tolist(), 3, TOL_F32, TIE_F32, True)
+    print(rep)
+    model.close()
+
+
+def test_long_prompt_many_attention_splits_bf16():
+    shape = inputs.get_shape("small_bf16").with_(prompt_len=333)
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    model, orc = _setup(shape, topo)
+    rep = run_parity(model, orc, shape, topo, inputs.make_prompt(shape).tolist(), 3, TOL_BF16, TIE_BF16, True,
+                     kv_check_layers=(0, 1, 2))
+    print(rep)
+    model.close()

@@ -391,3 +391,24 @@ def test_sal_cache_equals_one_shot():
         assert len(a.k) == len(b.k) == len(seq)
         for s in range(len(seq)):
             assert torch.allclose(a.k[s], b.k[s], atol=1e-9) and torch.allclose(a.v[s], b.v[s], atol=1e-9)
+
+
+def test_storage_rounding_mode_is_identity_without_rounding_and_small_with_bf16():
+    """storage=float64 rounds nothing: bit-identical to the plain oracle.  bf16 storage perturbs the
+    logits only at the bf16 level (it never changes the structure of the computation)."""
+    shape = MICRO
+    w = inputs.make_weights(shape, seed=0, std=0.2)
+    prompt = inputs.make_prompt(shape).tolist()
+    t = _tables(inputs.make_tree(shape.n_nodes, shape.topk))
+    outs = []
+    for storage in (None, torch.float64, torch.bfloat16):
+        orc = ao.Oracle(shape, w, dtype=torch.float64, storage=storage)
+        st = orc.prefill(prompt)
+        taps = {}
+        orc.step(st, t, None, taps)
+        outs.append((st.last_logits, taps["logits"], taps["d_logits"]))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    for a, c in zip(outs[0], outs[2]):
+        err = float((a - c).abs().max()) / max(1.0, float(a.abs().max()))
+        assert 0.0 < err < 3e-2
