@@ -24,6 +24,7 @@ class Report:
     max_logit_err: float = 0.0
     max_hidden_err: float = 0.0
     max_dlogit_err: float = 0.0
+    max_draft_err: float = 0.0
     max_kv_err: float = 0.0
     topk_tie_swaps: int = 0
     argmax_near_ties: int = 0
@@ -67,8 +68,11 @@ def compare_topk(shape, g_ids, g_vals, o_dlogits, tie_tol, rep: Report):
 
 
 def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int, tol: float,
-               tie_tol: float, planted: bool, kv_check_layers=(0, -1)) -> Report:
-    """model: paper_2406_13170_b200.Amphista.  Returns the error report; raises on a mismatch."""
+               tie_tol: float, planted: bool, kv_check_layers=(0, -1), tol_draft: Optional[float] = None) -> Report:
+    """model: paper_2406_13170_b200.Amphista.  Returns the error report; raises on a mismatch.
+    tol bounds the target's tensors, tol_draft (default: tol) those of the draft module."""
+    if tol_draft is None:
+        tol_draft = tol
     dev = model.device
     t = ao.tree_tables(topo.parent, topo.depth, topo.rank)
     N, K, d, V = t.n_nodes, shape.K, shape.d_model, shape.vocab
@@ -114,11 +118,13 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
         g_dl = model.get_tensor("d_logits", (K, V))
         scale = max(1.0, float(taps["d_logits"].abs().max()))
         rep.max_dlogit_err = max(rep.max_dlogit_err, rel_err(g_dl, taps["d_logits"]))
-        assert rel_err(g_dl, taps["d_logits"]) <= tol, f"step {i}: draft logits off by {rel_err(g_dl, taps['d_logits'])}"
-        assert rel_err(model.get_tensor("hp", (K, d)), taps["Hp"]) <= tol
-        assert rel_err(model.get_tensor("attn_o", (K, d)), taps["attn_o"]) <= tol
+        assert rel_err(g_dl, taps["d_logits"]) <= tol_draft, f"step {i}: draft logits off by {rel_err(g_dl, taps['d_logits'])}"
+        e_hp = rel_err(model.get_tensor("hp", (K, d)), taps["Hp"])
+        e_ao = rel_err(model.get_tensor("attn_o", (K, d)), taps["attn_o"])
         sal_h = model.get_tensor("sal_h", (2, d))
-        assert rel_err(sal_h[0], taps["h1"]) <= tol and rel_err(sal_h[1], taps["h2"]) <= tol
+        e_h1, e_h2 = rel_err(sal_h[0], taps["h1"]), rel_err(sal_h[1], taps["h2"])
+        rep.max_draft_err = max(rep.max_draft_err, e_hp, e_ao, e_h1, e_h2)
+        assert max(e_hp, e_ao, e_h1, e_h2) <= tol_draft, f"step {i}: draft hidden states off by {(e_h1, e_h2, e_hp, e_ao)}"
         # two candidates can only trade places if their oracle values are closer than twice the
         # measured error of the draft logits (itself bounded by tol above), or than the stated tie width
         e_abs = float((g_dl.to(torch.float64).cpu() - taps["d_logits"].to(torch.float64)).abs().max())
@@ -179,5 +185,5 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
             rows = model.get_tensor(f"sal{s+1}.{which}", (n_rows, d))
             e = rel_err(rows, torch.stack(cache))
             rep.max_kv_err = max(rep.max_kv_err, e)
-            assert e <= tol, f"stage {s+1} {which} cache off by {e}"
+            assert e <= tol_draft, f"stage {s+1} {which} cache off by {e}"
     return rep
