@@ -31,9 +31,9 @@ def tol_draft(n_layers: int) -> float:
     """The draft module sits on top of the target's last hidden state and adds two decoder layers, the head
     MLPs, the attention block and an un-normalised vocabulary projection (draft logits of a random-init
     model have a standard deviation of 11 against 1.3 for the target): the same storage rounding is amplified
-    further.  Measured on 7B widths against the plain oracle: 6e-2 on a 2-layer target, 0.11 on 8 layers, 0.40
+    further.  Measured on 7B widths against the plain oracle: 6e-2 to 0.12 on a 2-layer target (it varies with the prompt), 0.11 on 8 layers, 0.40
     on 32 layers, where the comparison stops being informative; it is then only bounded loosely."""
-    return 4.0 * tol_plain(n_layers) if n_layers <= 8 else 0.6
+    return 8.0 * tol_plain(n_layers) if n_layers <= 8 else 0.6
 
 
 def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1), storage=None):
