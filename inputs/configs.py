@@ -54,6 +54,10 @@ SHAPES = {
                              topk=(6, 5, 4, 3), n_nodes=32, prompt_len=48, steps=8),
     "7b": ModelShape("7b", 32, 4096, 32, 128, 11008, 32000, "bf16",
                      n_nodes=64, prompt_len=512, steps=128),
+    # 7B widths with two target layers and a 2048-token prompt: a few GB on the device, used for
+    # multi-pass profiler captures of single kernels at realistic sizes.
+    "7b_l2": ModelShape("7b_l2", 2, 4096, 32, 128, 11008, 32000, "bf16",
+                        n_nodes=64, prompt_len=2048, steps=8),
     "13b": ModelShape("13b", 40, 5120, 40, 128, 13824, 32000, "bf16",
                       n_nodes=64, prompt_len=1024, steps=128),
     "33b": ModelShape("33b", 60, 6656, 52, 128, 17920, 32000, "bf16",

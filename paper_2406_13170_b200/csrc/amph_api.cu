@@ -40,7 +40,7 @@ struct Layout {
   size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
-  size_t partial, att_o, att_ml, logits, d_logits;
+  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
   size_t partial_floats;
   int attn_splits;
 };
@@ -226,6 +226,8 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.att_ml = l.take(4 * (size_t)splits * c.n_heads * Mcap * 2);
   l.logits = l.take(4 * (size_t)Mcap * V);
   l.d_logits = l.take(4 * (size_t)kMaxK * V);
+  l.ss_a = l.take(4 * (size_t)Mcap * 32);
+  l.ss_b = l.take(4 * (size_t)Mcap * 32);
   *L = l;
   *Mcap_out = Mcap;
   const size_t per_layer = 2 * (size_t)c.n_heads * c.max_ctx * c.head_dim * esz;
@@ -336,17 +338,30 @@ PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg,
   return pv;
 }
 
-// One decoder layer over the rows described by `meta`.  On entry xn holds RMSNorm(x) * attn_norm;
-// on exit x is updated and, if next_gain is given, xn (and hid) hold RMSNorm(x) * next_gain.
-void layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
-                   int rows, int ctx_hi, const void* next_gain, float* hid) {
+RowScale row_scale_of(const amph_ctx* ctx, size_t off) {
+  RowScale rs;
+  rs.ss = ctx->at<float>(off);
+  rs.chunks = (ctx->cfg.d_model + kScaleChunkCols - 1) / kScaleChunkCols;
+  rs.d = ctx->cfg.d_model;
+  rs.eps = ctx->cfg.rms_eps;
+  return rs;
+}
+
+// One decoder layer over the rows described by `meta`.
+// Entry: xn holds the input of the q/k/v projections: attn_norm * x / rms(x) if !entry_deferred, else
+// attn_norm * x with the row sums of squares in ss_a (the division is applied after the projection).
+// Exit: x is updated.  With next_gain and no hid: xn = next_gain * x, sums of squares in ss_a (deferred form
+// for the next layer; returns true).  With hid: xn and hid hold the normalised rows (returns false).
+bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
+                   int rows, int ctx_hi, const void* next_gain, float* hid, bool entry_deferred) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
   PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
-  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st);
+  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st,
+                  entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale());
   }
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
@@ -356,19 +371,22 @@ void layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_NORM);
-  launch_resid_norm(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows, c.d_model, st);
+  launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st);
   }
   const void* gu[2] = {w.w_gate, w.w_up};
   P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
-  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st);
+  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b));
   }
   const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
-  { ProfScope ps(ctx, AMPH_PROF_NORM);
-  launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, next_gain ? ctx->ws + l.xn : nullptr, hid, c.rms_eps, rows,
-                    c.d_model, st);
+  ProfScope ps(ctx, AMPH_PROF_NORM);
+  if (hid != nullptr) {
+    launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, hid, c.rms_eps, rows, c.d_model, st);
+    return false;
   }
+  launch_resid_scale(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_a), rows, c.d_model, st);
+  return next_gain != nullptr;
 }
 
 // Target forward of the rows in `tok` under meta_v; leaves post-final-norm rows in hidden and xn.
@@ -390,10 +408,12 @@ void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
   launch_resid_norm(x, none, 0, 0, ctx->layers[0].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                     c.d_model, st);
   }
+  bool deferred = false;
   for (int i = 0; i < c.n_layers; ++i) {
     const bool last = i + 1 == c.n_layers;
-    layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
-                  last ? ctx->final_norm : ctx->layers[i + 1].attn_norm, last ? ctx->at<float>(l.hidden) : nullptr);
+    deferred = layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
+                             last ? ctx->final_norm : ctx->layers[i + 1].attn_norm,
+                             last ? ctx->at<float>(l.hidden) : nullptr, deferred);
   }
 }
 
@@ -429,7 +449,7 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
     }
-    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr);
+    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr, false);
     in_feat = hbuf;
   }
 }

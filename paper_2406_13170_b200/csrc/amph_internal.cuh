@@ -91,6 +91,16 @@ struct PartialView {
   size_t split_stride;      // floats between consecutive splits
 };
 
+// Deferred RMSNorm: a projection may be fed g * x (not yet divided by the row's RMS); the kernel that
+// consumes the projection's output multiplies by 1 / sqrt(sum_c ss[row][c] / d + eps).  ss == NULL: no scaling.
+struct RowScale {
+  const float* ss = nullptr;   // [rows][chunks] partial sums of squares of the row
+  int chunks = 0;
+  int d = 1;
+  float eps = 0.f;
+};
+constexpr int kScaleChunkCols = 512;     // columns per block of resid_scale_kernel (128 threads x float4)
+
 // ---- launchers (one per kernel family); dtype = AMPH_DTYPE_* of weights / activations / cache
 void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d,
                   float* x, cudaStream_t st);
@@ -101,12 +111,18 @@ void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, in
 void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype,
                        void* xn, float* hid, float eps, int rows, int d, cudaStream_t st);
 
+// Fully parallel variant for the inner layers: x <- x + sum P (mode 1) or sum P (mode 2); xn <- gain * x
+// (not normalised) and ss_part[row][chunk] <- sum of squares of the chunk.  gain == NULL: x only.
+void launch_resid_scale(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype, void* xn,
+                        float* ss_part, int rows, int d, cudaStream_t st);
+
 void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
                        cudaStream_t st);
 
 // q <- rope(sum P[:, 0:d]); K cache <- rope(sum P[:, d:2d]); V cache <- sum P[:, 2d:3d]
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv,
-                     int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st);
+                     int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st,
+                     RowScale rs = RowScale());
 
 struct AttnScratch {
   float* o;                 // [splits][heads][rows][head_dim]
@@ -119,7 +135,7 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
                                int head_dim, int max_ctx, int splits, cudaStream_t st);
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st);
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale());
 
 // cat[r] = [feat[r] ; tok_emb[next[r]]]   (Eq. 1's concatenation)
 void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat,

@@ -54,6 +54,13 @@ __device__ __forceinline__ float4 load4(const bf16* p) {
                      __uint_as_float(u.y & 0xffff0000u));
 }
 
+__device__ __forceinline__ float row_scale(const RowScale& rs, int row) {
+  if (rs.ss == nullptr) return 1.0f;
+  float tot = 0.f;
+  for (int c = 0; c < rs.chunks; ++c) tot += rs.ss[row * rs.chunks + c];       // fixed order
+  return 1.0f / sqrtf(tot / (float)rs.d + rs.eps);
+}
+
 __device__ __forceinline__ float block_sum(float v, float* red) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   const int w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
@@ -138,6 +145,41 @@ void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const voi
                            x, P, col_off, mode, (const T*)gain, (T*)xn, hid, eps, d));
 }
 
+// Residual update without the row-wide reduction: grid (row, 512-column chunk).  The division by the row's
+// RMS is left to the kernel that consumes the next projection (RowScale), so every block is independent.
+template <typename T>
+__global__ void __launch_bounds__(128)
+resid_scale_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, const T* __restrict__ gain,
+                   T* __restrict__ xn, float* __restrict__ ss_part, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const int c = blockIdx.y * kScaleChunkCols + threadIdx.x * 4;
+  float ss = 0.f;
+  if (c < d) {
+    float* xr = x + (size_t)r * d + c;
+    float4 v = sum_partials4(P, r, col_off + c);
+    if (mode == 1) { const float4 o = load4(xr); v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+    store4(xr, v);
+    if (gain != nullptr) {
+      const float4 g = load4(gain + c);
+      store4(xn + (size_t)r * d + c, make_float4(g.x * v.x, g.y * v.y, g.z * v.z, g.w * v.w));
+      ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  }
+  if (gain == nullptr) return;
+  const float tot = block_sum(ss, red);
+  if (threadIdx.x == 0) ss_part[r * gridDim.y + blockIdx.y] = tot;
+}
+
+void launch_resid_scale(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype, void* xn,
+                        float* ss_part, int rows, int d, cudaStream_t st) {
+  const int chunks = (d + kScaleChunkCols - 1) / kScaleChunkCols;
+  AMPH_DISPATCH(dtype, launch_pdl(resid_scale_kernel<T>, dim3(rows, chunks), dim3(128), 0, st, x, P, col_off, mode,
+                                  (const T*)gain, (T*)xn, ss_part, d));
+}
+
 // --------------------------------------------------------------------------------------------
 // rotary table for the rows of one call: table[r][i] = (cos, sin)(pos[r] * theta^(-2i/dh))
 // --------------------------------------------------------------------------------------------
@@ -163,9 +205,9 @@ void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* tabl
 // q / k rotation, KV-cache write (one block per row)
 // --------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(256)
 qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* __restrict__ rope, T* __restrict__ q,
-                T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx) {
+                T* __restrict__ kc, T* __restrict__ vc, int n_heads, int dh, int max_ctx, RowScale rs) {
   pdl_wait();
   pdl_launch_dependents();
   const int r = blockIdx.x;
@@ -173,37 +215,43 @@ qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* _
   const bool live = r < meta->n_rows;
   const int slot = meta->slot[r];
   const bool store = live && slot >= 0 && slot < max_ctx;
-  for (int idx = threadIdx.x; idx < n_heads * quads; idx += blockDim.x) {
-    const int h = idx / quads, i = (idx - h * quads) * 4;          // four rotation pairs (i..i+3, i+half..)
+  const float sc = row_scale(rs, r);
+  // one item = four rotation pairs (i..i+3, i+half..) of one head; grid.y strides over the items of the row
+  for (int idx = blockIdx.y * blockDim.x + threadIdx.x; idx < n_heads * quads; idx += gridDim.y * blockDim.x) {
+    const int h = idx / quads, i = (idx - h * quads) * 4;
     const float4 cs0 = *reinterpret_cast<const float4*>(rope + r * half + i);       // (c0,s0,c1,s1)
     const float4 cs1 = *reinterpret_cast<const float4*>(rope + r * half + i + 2);   // (c2,s2,c3,s3)
     const int c0 = h * dh + i, c1 = c0 + half;
     {
-      const float4 a = sum_partials4(P, r, c0), b = sum_partials4(P, r, c1);
+      float4 a = sum_partials4(P, r, c0), b = sum_partials4(P, r, c1);
+      a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
       store4(q + (size_t)r * d + c0, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
                                                  a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
       store4(q + (size_t)r * d + c1, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
                                                  b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
     }
     if (store) {
-      const float4 a = sum_partials4(P, r, d + c0), b = sum_partials4(P, r, d + c1);
+      float4 a = sum_partials4(P, r, d + c0), b = sum_partials4(P, r, d + c1);
+      a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
       const size_t o = ((size_t)h * max_ctx + slot) * dh + i;
       store4(kc + o, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
                                  a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
       store4(kc + o + half, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
                                         b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
-      store4(vc + o, sum_partials4(P, r, 2 * d + c0));
-      store4(vc + o + half, sum_partials4(P, r, 2 * d + c1));
+      float4 v0 = sum_partials4(P, r, 2 * d + c0), v1 = sum_partials4(P, r, 2 * d + c1);
+      store4(vc + o, make_float4(v0.x * sc, v0.y * sc, v0.z * sc, v0.w * sc));
+      store4(vc + o + half, make_float4(v1.x * sc, v1.y * sc, v1.z * sc, v1.w * sc));
     }
   }
 }
 
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv, int dtype,
-                     int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st) {
-  int threads = (n_heads * head_dim / 8 + 31) / 32 * 32;
-  if (threads > 1024) threads = 1024;
-  AMPH_DISPATCH(dtype, launch_pdl(qkv_rope_kernel<T>, dim3(rows), dim3(threads), 0, st, P, meta, rope, (T*)q, (T*)kv.k, (T*)kv.v,
-                                                                    n_heads, head_dim, max_ctx));
+                     int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st, RowScale rs) {
+  const int items = n_heads * head_dim / 8;
+  const int threads = items >= 128 ? 128 : (items + 31) / 32 * 32;
+  const int gy = (items + threads - 1) / threads;
+  AMPH_DISPATCH(dtype, launch_pdl(qkv_rope_kernel<T>, dim3(rows, gy), dim3(threads), 0, st, P, meta, rope, (T*)q,
+                                  (T*)kv.k, (T*)kv.v, n_heads, head_dim, max_ctx, rs));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -403,22 +451,28 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 // SwiGLU on the fused gate / up projection: act = silu(gate) * up
 // --------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f) {
+__global__ void __launch_bounds__(256)
+swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f, RowScale rs) {
   pdl_wait();
   pdl_launch_dependents();
-  const size_t n = (size_t)rows * f;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    const int r = (int)(i / f), c = (int)(i - (size_t)r * f);
-    const float g = sum_partials(P, r, c), u = sum_partials(P, r, f + c);
-    act[i] = from_f<T>(g / (1.0f + expf(-g)) * u);
+  const int r = blockIdx.x;
+  const float sc = row_scale(rs, r);
+  for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < f; c += gridDim.y * blockDim.x * 4) {
+    const float4 g = sum_partials4(P, r, c), u = sum_partials4(P, r, f + c);
+    float4 o;
+    float t;
+    t = g.x * sc; o.x = t / (1.0f + expf(-t)) * (u.x * sc);
+    t = g.y * sc; o.y = t / (1.0f + expf(-t)) * (u.y * sc);
+    t = g.z * sc; o.z = t / (1.0f + expf(-t)) * (u.z * sc);
+    t = g.w * sc; o.w = t / (1.0f + expf(-t)) * (u.w * sc);
+    store4(act + (size_t)r * f + c, o);
   }
 }
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st) {
-  const size_t n = (size_t)rows * f;
-  int blocks = (int)((n + 255) / 256);
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, P, (T*)act, rows, f));
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs) {
+  int gy = (f / 4 + 255) / 256;
+  if (gy > 16) gy = 16;
+  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(rows, gy), dim3(256), 0, st, P, (T*)act, rows, f, rs));
 }
 
 // --------------------------------------------------------------------------------------------
