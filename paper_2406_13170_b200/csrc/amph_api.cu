@@ -75,6 +75,8 @@ struct amph_ctx {
   int ctx_hi;               // host-side upper bound of the committed length
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
+  int sm_count = 148;
+  bool last_proj_one_wave = false;   // the last projection ran on the tensor-core kernel with a fully resident grid
   cudaGraphExec_t graph_exec = nullptr;   // captured draft -> verify -> accept schedule of amph_step
   int graph_key = -1;       // attention split counts the captured grids were sized for
   bool graph_off = false;   // capture is not possible (legacy stream, flag) or failed once
@@ -316,11 +318,13 @@ PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int 
 PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
   float* P = ctx->at<float>(ctx->lay.partial);
   PartialView pv;
+  ctx->last_proj_one_wave = false;
   if (ctx->tc) {
     int splits = 0;
     size_t stride = 0;
     if (tc_gemm_launch(ctx->tc, xb, w, n_seg, out, in, rows, P, ctx->lay.partial_floats, &splits, &stride,
                        ctx->stream)) {
+      ctx->last_proj_one_wave = (long long)n_seg * (out / 128) * splits <= 2LL * ctx->sm_count;
       pv.p = P;
       pv.splits = splits;
       pv.ld = n_seg * out;
@@ -366,17 +370,18 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
   launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
-                        c.max_ctx, ctx_hi, l.attn_splits, st);
+                        c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr);
   }
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_NORM);
-  launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st);
+  launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st,
+                     ctx->last_proj_one_wave);
   }
   const void* gu[2] = {w.w_gate, w.w_up};
   P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
-  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b));
+  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b), ctx->last_proj_one_wave);
   }
   const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
@@ -385,7 +390,8 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
     launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, hid, c.rms_eps, rows, c.d_model, st);
     return false;
   }
-  launch_resid_scale(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_a), rows, c.d_model, st);
+  launch_resid_scale(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_a), rows, c.d_model, st,
+                     ctx->last_proj_one_wave && next_gain != nullptr);
   return next_gain != nullptr;
 }
 
@@ -623,6 +629,7 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   ctx->phase = PH_CREATED;
   ctx->ctx_hi = 0;
   ctx->tc = nullptr;
+  { int dv = 0; cudaGetDevice(&dv); cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dv); }
   const size_t half_layer = (size_t)cfg->n_heads * cfg->max_ctx * cfg->head_dim * ctx->esz;
   ctx->kv_target.resize(cfg->n_layers);
   char* p = ctx->kv;

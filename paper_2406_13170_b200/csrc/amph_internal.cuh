@@ -113,8 +113,11 @@ void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const voi
 
 // Fully parallel variant for the inner layers: x <- x + sum P (mode 1) or sum P (mode 2); xn <- gain * x
 // (not normalised) and ss_part[row][chunk] <- sum of squares of the chunk.  gain == NULL: x only.
+// early != 0: let the next kernel (a projection, which only prefetches weights until its own wait) start
+// launching before this kernel has waited for its predecessor.  The caller sets it only when the
+// predecessor's grid is fully resident (one wave), so that the early starter cannot take its slots.
 void launch_resid_scale(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype, void* xn,
-                        float* ss_part, int rows, int d, cudaStream_t st);
+                        float* ss_part, int rows, int d, cudaStream_t st, int early = 0);
 
 void launch_rope_table(const RowMeta* meta, const double* inv_freq, float2* table, int rows, int half,
                        cudaStream_t st);
@@ -130,12 +133,13 @@ struct AttnScratch {
 };
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out,
                            int dtype, int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi,
-                           int max_splits, cudaStream_t st);
+                           int max_splits, cudaStream_t st, int early = 0);
 
 void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
                                int head_dim, int max_ctx, int splits, cudaStream_t st);
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale());
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale(),
+                   int early = 0);
 
 // cat[r] = [feat[r] ; tok_emb[next[r]]]   (Eq. 1's concatenation)
 void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat,

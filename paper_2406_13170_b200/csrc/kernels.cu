@@ -150,9 +150,10 @@ void launch_resid_norm(float* x, PartialView P, int col_off, int mode, const voi
 template <typename T>
 __global__ void __launch_bounds__(128)
 resid_scale_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, const T* __restrict__ gain,
-                   T* __restrict__ xn, float* __restrict__ ss_part, int d) {
+                   T* __restrict__ xn, float* __restrict__ ss_part, int d, int early) {
+  if (early) pdl_launch_dependents();
   pdl_wait();
-  pdl_launch_dependents();
+  if (!early) pdl_launch_dependents();
   __shared__ float red[32];
   const int r = blockIdx.x;
   const int c = blockIdx.y * kScaleChunkCols + threadIdx.x * 4;
@@ -174,10 +175,10 @@ resid_scale_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, 
 }
 
 void launch_resid_scale(float* x, PartialView P, int col_off, int mode, const void* gain, int dtype, void* xn,
-                        float* ss_part, int rows, int d, cudaStream_t st) {
+                        float* ss_part, int rows, int d, cudaStream_t st, int early) {
   const int chunks = (d + kScaleChunkCols - 1) / kScaleChunkCols;
   AMPH_DISPATCH(dtype, launch_pdl(resid_scale_kernel<T>, dim3(rows, chunks), dim3(128), 0, st, x, P, col_off, mode,
-                                  (const T*)gain, (T*)xn, ss_part, d));
+                                  (const T*)gain, (T*)xn, ss_part, d, early));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -391,9 +392,10 @@ tree_attn_kernel(const T* __restrict__ q, const T* __restrict__ kc, const T* __r
 
 template <typename T>
 __global__ void attn_combine_kernel(const float* __restrict__ po, const float* __restrict__ pml,
-                                    T* __restrict__ out, int splits, int rows_cap, int n_heads, int dh) {
+                                    T* __restrict__ out, int splits, int rows_cap, int n_heads, int dh, int early) {
+  if (early) pdl_launch_dependents();
   pdl_wait();
-  pdl_launch_dependents();
+  if (!early) pdl_launch_dependents();
   const int r = blockIdx.x, h = blockIdx.y;
   float M = -INFINITY;
   for (int s = 0; s < splits; ++s)
@@ -425,19 +427,19 @@ static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, Attn
   launch_pdl(tree_attn_kernel<T, DH>, dim3(grid), dim3(kAttThreads), smem, st, (const T*)q, (const T*)kv.k, (const T*)kv.v, meta,
                                                           sc.o, sc.ml, rows, n_heads, max_ctx);
   launch_pdl(attn_combine_kernel<T>, dim3(dim3(rows, n_heads)), dim3(DH < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (T*)out, splits, rows,
-                                                                              n_heads, DH);
+                                                                              n_heads, DH, 0);
 }
 
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out, int dtype,
                            int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi, int max_splits,
-                           cudaStream_t st) {
+                           cudaStream_t st, int early) {
   int splits = (ctx_hi + 127) / 128;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
   if (dtype == AMPH_DTYPE_BF16) {                    // tensor-core path; the kernel below serves fp32 caches
     launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st);
     launch_pdl(attn_combine_kernel<bf16>, dim3(dim3(rows, n_heads)), dim3(head_dim < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (bf16*)out, splits,
-                                                                                        rows, n_heads, head_dim);
+                                                                                        rows, n_heads, head_dim, early);
     return;
   }
   if (head_dim == 64) {
@@ -452,9 +454,10 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 // --------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
-swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f, RowScale rs) {
+swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f, RowScale rs, int early) {
+  if (early) pdl_launch_dependents();
   pdl_wait();
-  pdl_launch_dependents();
+  if (!early) pdl_launch_dependents();
   const int r = blockIdx.x;
   const float sc = row_scale(rs, r);
   for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < f; c += gridDim.y * blockDim.x * 4) {
@@ -469,10 +472,10 @@ swiglu_kernel(PartialView P, T* __restrict__ act, int rows, int f, RowScale rs) 
   }
 }
 
-void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs) {
+void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs, int early) {
   int gy = (f / 4 + 255) / 256;
   if (gy > 16) gy = 16;
-  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(rows, gy), dim3(256), 0, st, P, (T*)act, rows, f, rs));
+  AMPH_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(rows, gy), dim3(256), 0, st, P, (T*)act, rows, f, rs, early));
 }
 
 // --------------------------------------------------------------------------------------------
