@@ -332,7 +332,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   // K-splits: fill about two CTAs per SM, keep at least four 64-wide K blocks per CTA
   int splits = (2 * g->sm_count) / tiles;
   if (splits > kblocks / 4) splits = kblocks / 4;
-  if (splits > 8) splits = 8;                             // consumers fetch up to eight partial sums at once
+  if (splits > 16) splits = 16;
   while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
   if (splits < 1) splits = 1;
   if ((size_t)nt * ld > p_floats) return false;

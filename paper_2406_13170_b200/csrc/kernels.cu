@@ -28,19 +28,13 @@ __device__ __forceinline__ float sum_partials(const PartialView& P, int row, int
   return acc;
 }
 
-// Same for four consecutive columns.  The loads of up to eight splits are issued before any is consumed
-// (the partial sums sit in L2 slices that may be a microsecond away); the additions keep the split order.
 __device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, int col) {
   const float* p = P.p + (size_t)row * P.ld + col;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < P.splits; s0 += 8) {
-    float4 v[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (s0 + i < P.splits) v[i] = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(s0 + i) * P.split_stride));
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (s0 + i < P.splits) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
+  float4 acc = *reinterpret_cast<const float4*>(p);
+#pragma unroll 4
+  for (int s = 1; s < P.splits; ++s) {
+    const float4 v = *reinterpret_cast<const float4*>(p + (size_t)s * P.split_stride);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
   return acc;
 }
