@@ -84,12 +84,14 @@ __global__ void embed_kernel(const T* __restrict__ emb, const int* __restrict__ 
   int t = toks[r];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
   const T* e = emb + (size_t)t * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)r * d + c] = to_f(e[c]);
+  for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < d; c += gridDim.y * blockDim.x * 4)
+    store4(x + (size_t)r * d + c, load4(e + c));
 }
 
 void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d, float* x,
                   cudaStream_t st) {
-  AMPH_DISPATCH(dtype, launch_pdl(embed_kernel<T>, dim3(rows), dim3(256), 0, st, (const T*)tok_emb, toks, vocab, d, x));
+  const int gy = (d / 4 + 255) / 256;
+  AMPH_DISPATCH(dtype, launch_pdl(embed_kernel<T>, dim3(rows, gy), dim3(256), 0, st, (const T*)tok_emb, toks, vocab, d, x));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -489,15 +491,16 @@ __global__ void concat_kernel(const float* __restrict__ feat, const T* __restric
   const int r = blockIdx.x;
   int t = next_tok[r];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    cat[(size_t)r * 2 * d + c] = from_f<T>(feat[(size_t)r * d + c]);
-    cat[(size_t)r * 2 * d + d + c] = emb[(size_t)t * d + c];
+  for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < d; c += gridDim.y * blockDim.x * 4) {
+    store4(cat + (size_t)r * 2 * d + c, load4(feat + (size_t)r * d + c));
+    store4(cat + (size_t)r * 2 * d + d + c, load4(emb + (size_t)t * d + c));
   }
 }
 
 void launch_concat(const float* feat, const void* tok_emb, const int* next_tok, int vocab, void* cat, int dtype,
                    int rows, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, launch_pdl(concat_kernel<T>, dim3(rows), dim3(256), 0, st, feat, (const T*)tok_emb, next_tok, vocab, (T*)cat, d));
+  const int gy = (d / 4 + 255) / 256;
+  AMPH_DISPATCH(dtype, launch_pdl(concat_kernel<T>, dim3(rows, gy), dim3(256), 0, st, feat, (const T*)tok_emb, next_tok, vocab, (T*)cat, d));
 }
 
 // --------------------------------------------------------------------------------------------
@@ -584,16 +587,17 @@ __global__ void gather_last_kernel(const float* __restrict__ h1, const float* __
   int lr = s->n_pending - 1;
   lr = lr < 0 ? 0 : (lr >= kPendMax ? kPendMax - 1 : lr);
   const float* src = blockIdx.x == 0 ? h1 : h2;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float v = src[(size_t)lr * d + c];
-    last[(size_t)blockIdx.x * d + c] = v;
-    last_act[(size_t)blockIdx.x * d + c] = from_f<T>(v);
+  for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < d; c += gridDim.y * blockDim.x * 4) {
+    const float4 v = load4(src + (size_t)lr * d + c);
+    store4(last + (size_t)blockIdx.x * d + c, v);
+    store4(last_act + (size_t)blockIdx.x * d + c, v);
   }
 }
 
 void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev, float* last, void* last_act,
                         int dtype, int d, cudaStream_t st) {
-  AMPH_DISPATCH(dtype, launch_pdl(gather_last_kernel<T>, dim3(2), dim3(256), 0, st, h1, h2, st_dev, last, (T*)last_act, d));
+  const int gy = (d / 4 + 255) / 256;
+  AMPH_DISPATCH(dtype, launch_pdl(gather_last_kernel<T>, dim3(2, gy), dim3(256), 0, st, h1, h2, st_dev, last, (T*)last_act, d));
 }
 
 struct BiasPtrs { const void* b[kMaxK]; };
@@ -607,12 +611,18 @@ __global__ void mlp_heads_kernel(PartialView P, const float* __restrict__ last, 
   const int k = blockIdx.x;
   const int row = (k < K / 2 || n_sal == 1) ? 0 : 1;       // Eq. 2: first half of the heads <- stage 1
   const T* b = (const T*)bias.b[k];
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float pre = sum_partials(P, row, k * d + c) + to_f(b[c]);
-    const float v = last[(size_t)row * d + c] + pre / (1.0f + expf(-pre)) + to_f(pe[(size_t)k * d + c]);
-    hp[(size_t)k * d + c] = v;
-    ao[(size_t)k * d + c] = v;                // the attention block updates this copy in place
-    ao_act[(size_t)k * d + c] = from_f<T>(v);
+  for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < d; c += gridDim.y * blockDim.x * 4) {
+    const float4 w = sum_partials4(P, row, k * d + c), bb = load4(b + c), l = load4(last + (size_t)row * d + c),
+                 e = load4(pe + (size_t)k * d + c);
+    float4 v;
+    float pre;
+    pre = w.x + bb.x; v.x = l.x + pre / (1.0f + expf(-pre)) + e.x;
+    pre = w.y + bb.y; v.y = l.y + pre / (1.0f + expf(-pre)) + e.y;
+    pre = w.z + bb.z; v.z = l.z + pre / (1.0f + expf(-pre)) + e.z;
+    pre = w.w + bb.w; v.w = l.w + pre / (1.0f + expf(-pre)) + e.w;
+    store4(hp + (size_t)k * d + c, v);
+    store4(ao + (size_t)k * d + c, v);          // the attention block updates this copy in place
+    store4(ao_act + (size_t)k * d + c, v);
   }
 }
 
@@ -620,7 +630,8 @@ void launch_mlp_heads(PartialView P, const float* last, const void* const* bias,
                       float* ao, void* ao_act, int dtype, int K, int n_sal, int d, cudaStream_t st) {
   BiasPtrs bp;
   for (int k = 0; k < kMaxK; ++k) bp.b[k] = k < K ? bias[k] : nullptr;
-  AMPH_DISPATCH(dtype, launch_pdl(mlp_heads_kernel<T>, dim3(K), dim3(256), 0, st, P, last, bp, (const T*)pe, hp, ao, (T*)ao_act,
+  const int gy = (d / 4 + 127) / 128;
+  AMPH_DISPATCH(dtype, launch_pdl(mlp_heads_kernel<T>, dim3(K, gy), dim3(128), 0, st, P, last, bp, (const T*)pe, hp, ao, (T*)ao_act,
                                                               K, n_sal, d));
 }
 
@@ -629,17 +640,17 @@ template <typename T>
 __global__ void aeb_attention_kernel(PartialView P, T* __restrict__ out, int K, int n_heads, int dh) {
   pdl_wait();
   pdl_launch_dependents();
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
   float* qs = sm;                 // [K][dh]
   float* ks = qs + K * dh;
   float* vs = ks + K * dh;
   float* pr = vs + K * dh;        // [K][K]
   const int h = blockIdx.x, d = n_heads * dh;
-  for (int i = threadIdx.x; i < K * dh; i += blockDim.x) {
-    const int r = i / dh, c = i - r * dh;
-    qs[i] = sum_partials(P, r, h * dh + c);
-    ks[i] = sum_partials(P, r, d + h * dh + c);
-    vs[i] = sum_partials(P, r, 2 * d + h * dh + c);
+  const int per = K * dh / 4;                            // float4 items per q / k / v block
+  for (int i = threadIdx.x; i < 3 * per; i += blockDim.x) {
+    const int which = i / per, j = (i - which * per) * 4;
+    const int r = j / dh, c = j - r * dh;
+    store4(sm + which * K * dh + j, sum_partials4(P, r, which * d + h * dh + c));
   }
   __syncthreads();
   const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -700,15 +711,30 @@ __device__ void block_best(float& v, int& i, float* sv, int* si) {
 struct TopkCounts { int c[kMaxK]; };
 
 __global__ void topk_heads_kernel(PartialView P, int vocab, TopkCounts ck, int* __restrict__ ids,
-                                  float* __restrict__ vals, float* __restrict__ d_logits) {
+                                  float* __restrict__ vals, float* __restrict__ d_logits, int mode) {
   pdl_wait();
   pdl_launch_dependents();
+  extern __shared__ __align__(16) float rowbuf[];       // the head's logits when they fit, else the global copy is used
   __shared__ float sv[32];
   __shared__ int si[32];
   const int k = blockIdx.x;
-  float* row = d_logits + (size_t)k * vocab;
-  for (int c = threadIdx.x; c < vocab; c += blockDim.x) row[c] = sum_partials(P, k, k * vocab + c);
+  const int in_smem = mode & 1, vec = mode & 2;          // bit 0: row cached in shared memory; bit 1: 16-byte loads are aligned
+  float* grow = d_logits + (size_t)k * vocab;
+  for (int c = threadIdx.x * 4; c < vocab; c += blockDim.x * 4) {
+    if (vec && c + 3 < vocab) {
+      const float4 v = sum_partials4(P, k, k * vocab + c);
+      store4(grow + c, v);
+      if (in_smem) store4(rowbuf + c, v);
+    } else {
+      for (int e = c; e < vocab && e < c + 4; ++e) {
+        const float v = sum_partials(P, k, k * vocab + e);
+        grow[e] = v;
+        if (in_smem) rowbuf[e] = v;
+      }
+    }
+  }
   __syncthreads();
+  const float* row = in_smem ? rowbuf : grow;
   float pv = INFINITY;
   int pi = -1;
   for (int t = 0; t < ck.c[k]; ++t) {
@@ -730,7 +756,12 @@ void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids,
                        cudaStream_t st) {
   TopkCounts c;
   for (int k = 0; k < kMaxK; ++k) c.c[k] = k < K ? ck[k] : 0;
-  launch_pdl(topk_heads_kernel, dim3(K), dim3(1024), 0, st, P, vocab, c, ids, vals, d_logits);
+  const size_t bytes = (size_t)vocab * sizeof(float);
+  const int vec = vocab % 4 == 0 && P.ld % 4 == 0;
+  const int in_smem = bytes <= 200 * 1024;
+  if (in_smem) cudaFuncSetAttribute(topk_heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  launch_pdl(topk_heads_kernel, dim3(K), dim3(1024), in_smem ? bytes : 0, st, P, vocab, c, ids, vals, d_logits,
+             in_smem | (vec << 1));
 }
 
 __global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ amax,
