@@ -40,7 +40,7 @@ struct Layout {
   size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
-  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
+  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b, tc_counters;
   size_t partial_floats;
   int attn_splits;
 };
@@ -230,7 +230,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.d_logits = l.take(4 * (size_t)kMaxK * V);
   l.ss_a = l.take(4 * (size_t)Mcap * 128);
   l.ss_b = l.take(4 * (size_t)Mcap * 128);
-
+  l.tc_counters = l.take(sizeof(int) * kTcCounterInts);
   *L = l;
   *Mcap_out = Mcap;
   const size_t per_layer = 2 * (size_t)c.n_heads * c.max_ctx * c.head_dim * esz;
@@ -329,6 +329,7 @@ PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg,
   if (ctx->tc) {
     int splits = 0;
     size_t stride = 0;
+    if (epi) epi->counters = ctx->at<int>(ctx->lay.tc_counters);
     if (epi && fused && !(ctx->cfg.flags & AMPH_FLAG_NO_FUSED_EPILOGUE) &&
         tc_gemm_launch(ctx->tc, xb, w, n_seg, out, in, rows, P, ctx->lay.partial_floats, &splits, &stride,
                        ctx->stream, epi)) {

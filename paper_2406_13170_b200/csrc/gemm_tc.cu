@@ -130,33 +130,13 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// ---- thread-block cluster helpers (fused epilogues): the CTAs that hold the split-K partials of one tile
-// form a cluster and reduce through distributed shared memory.
-__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// float4 at shared-memory address `local` (an address of this CTA) in the CTA of rank `cta` of the cluster
-__device__ __forceinline__ float4 ld_dsmem4(uint32_t local, uint32_t cta) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(cta));
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
-  return v;
-}
-// Sum over the cluster's CTAs, in rank order, of the float4 at (row, 4 * lane) of their staged tiles
-// ([rows][128] fp32 at shared-memory offset `stage`).  All loads are issued before the additions.
-__device__ __forceinline__ float4 sum_cluster4(uint32_t stage, int row, int lane, int n_cta) {
-  const uint32_t a = stage + (uint32_t)(row * kTileM + 4 * lane) * 4u;
-  float4 v[8];
-#pragma unroll
-  for (int c = 0; c < 8; ++c)
-    if (c < n_cta) v[c] = ld_dsmem4(a, (uint32_t)c);
-  float4 acc = v[0];
-#pragma unroll
-  for (int c = 1; c < 8; ++c)
-    if (c < n_cta) { acc.x += v[c].x; acc.y += v[c].y; acc.z += v[c].z; acc.w += v[c].w; }
+__device__ __forceinline__ float4 sum_tile4(const TcParams& prm, int r, int col) {
+  const float* p = prm.P + (size_t)r * prm.ld + col;
+  float4 acc = __ldcg(reinterpret_cast<const float4*>(p));
+  for (int s = 1; s < prm.splits; ++s) {                         // split order: deterministic
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(p + (size_t)s * prm.split_stride));
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
   return acc;
 }
 __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
@@ -172,26 +152,23 @@ __device__ __forceinline__ float4 unpack4_bf16(const __nv_bfloat16* p) {
                      __uint_as_float(u.y & 0xffff0000u));
 }
 
-// Fused epilogue, run by the four epilogue warps (et = 0..127) of every CTA of the cluster after all of them
-// have staged their partial tile.  Each CTA finishes the rows r with r % n_cta == rank.  inv_s[r] is the
-// deferred RMS division of row r (1 when none).
-__device__ void fused_epilogue(const TcParams& prm, int tile, int et, const float* inv_s, uint32_t stage,
-                               int rank, int n_cta) {
+// Runs in the CTA that completed a tile: et = 0..127 indexes the four epilogue warps' threads,
+// inv_s[r] is the deferred RMS division of row r (1 when none).
+__device__ void fused_epilogue(const TcParams& prm, int tile, int et, const float* inv_s) {
   const TcEpilogue& e = prm.epi;
   typedef __nv_bfloat16 bf16;
   const int rows = prm.rows, tps = prm.tiles_per_seg;
   const int lane = et & 31, ew = et >> 5;
   if (e.mode == TC_EPI_RESIDUAL) {
     const int d = prm.ld, c = tile * kTileM + 4 * lane;
-    for (int r = rank + n_cta * ew; r < rows; r += n_cta * 4) {
+    for (int r = ew; r < rows; r += 4) {
+      float4 v = sum_tile4(prm, r, c);
       float* xr = e.x + (size_t)r * d + c;
       const float4 o = *reinterpret_cast<const float4*>(xr);
-      float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (e.gain != nullptr) g = unpack4_bf16(reinterpret_cast<const bf16*>(e.gain) + c);
-      float4 v = sum_cluster4(stage, r, lane, n_cta);
       v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
       *reinterpret_cast<float4*>(xr) = v;
       if (e.gain != nullptr) {
+        const float4 g = unpack4_bf16(reinterpret_cast<const bf16*>(e.gain) + c);
         *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.xn) + (size_t)r * d + c) =
             pack4_bf16(g.x * v.x, g.y * v.y, g.z * v.z, g.w * v.w);
         float ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -200,12 +177,10 @@ __device__ void fused_epilogue(const TcParams& prm, int tile, int et, const floa
       }
     }
   } else if (e.mode == TC_EPI_SWIGLU) {
-    // cluster of two: rank 0 holds the gate tile, rank 1 the up tile of the same 128 features (one K split)
     const int f = prm.ld / 2, c = (tile % tps) * kTileM + 4 * lane;
-    for (int r = rank + 2 * ew; r < rows; r += 8) {
-      const uint32_t a = stage + (uint32_t)(r * kTileM + 4 * lane) * 4u;
-      const float4 g = ld_dsmem4(a, 0u), u = ld_dsmem4(a, 1u);
+    for (int r = ew; r < rows; r += 4) {
       const float sc = inv_s[r];
+      const float4 g = sum_tile4(prm, r, c), u = sum_tile4(prm, r, f + c);
       float t0 = g.x * sc, t1 = g.y * sc, t2 = g.z * sc, t3 = g.w * sc;
       t0 = t0 / (1.0f + expf(-t0)) * (u.x * sc);
       t1 = t1 / (1.0f + expf(-t1)) * (u.y * sc);
@@ -214,33 +189,20 @@ __device__ void fused_epilogue(const TcParams& prm, int tile, int et, const floa
       *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.act) + (size_t)r * f + c) = pack4_bf16(t0, t1, t2, t3);
     }
   } else if (e.mode == TC_EPI_QKV_ROPE) {
-    // lane l < 16 of a warp takes the rotation pairs (4l..4l+3, +half) of the first row, lanes 16..31 the second row
     const int dh = e.head_dim, half = dh >> 1, quads = half >> 2, d = e.n_heads * dh;
     const int seg = tile / tps, feat0 = (tile - seg * tps) * kTileM;
-    const int item = lane & 15, sub = lane >> 4;
-    const int hh = item / quads, i4 = (item - hh * quads) * 4;
-    const int l0 = hh * dh + i4, l1 = l0 + half;               // columns inside the 128-wide tile
-    const int c0 = feat0 + l0, c1 = feat0 + l1;
+    const int item = et & 15, rsub = et >> 4;                  // 16 items (4 rotation pairs each) per row
+    const int hh = item / quads, i = (item - hh * quads) * 4;
+    const int c0 = feat0 + hh * dh + i, c1 = c0 + half;
     const int h = c0 / dh;
     const int n_rows = e.meta->n_rows;
-    for (int r = rank + n_cta * (2 * ew + sub); r < rows; r += n_cta * 8) {
-      const uint32_t a0 = stage + (uint32_t)(r * kTileM + l0) * 4u, a1 = stage + (uint32_t)(r * kTileM + l1) * 4u;
-      float4 va[8], vb[8];
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        if (c < n_cta) { va[c] = ld_dsmem4(a0, (uint32_t)c); vb[c] = ld_dsmem4(a1, (uint32_t)c); }
-      float4 a = va[0], b = vb[0];
-#pragma unroll
-      for (int c = 1; c < 8; ++c)
-        if (c < n_cta) {
-          a.x += va[c].x; a.y += va[c].y; a.z += va[c].z; a.w += va[c].w;
-          b.x += vb[c].x; b.y += vb[c].y; b.z += vb[c].z; b.w += vb[c].w;
-        }
+    for (int r = rsub; r < rows; r += 8) {
       const float sc = inv_s[r];
+      float4 a = sum_tile4(prm, r, seg * d + c0), b = sum_tile4(prm, r, seg * d + c1);
       a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
       const int slot = e.meta->slot[r];
       const bool store = r < n_rows && slot >= 0 && slot < e.max_ctx;
-      const size_t co = ((size_t)h * e.max_ctx + (store ? slot : 0)) * dh + i4;
+      const size_t co = ((size_t)h * e.max_ctx + (store ? slot : 0)) * dh + i;
       if (seg == 2) {
         if (store) {
           *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.vc) + co) = pack4_bf16(a.x, a.y, a.z, a.w);
@@ -248,8 +210,8 @@ __device__ void fused_epilogue(const TcParams& prm, int tile, int et, const floa
         }
         continue;
       }
-      const float4 cs0 = *reinterpret_cast<const float4*>(e.rope + r * half + i4);
-      const float4 cs1 = *reinterpret_cast<const float4*>(e.rope + r * half + i4 + 2);
+      const float4 cs0 = *reinterpret_cast<const float4*>(e.rope + r * half + i);
+      const float4 cs1 = *reinterpret_cast<const float4*>(e.rope + r * half + i + 2);
       const uint2 lo = pack4_bf16(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
                                   a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w);
       const uint2 hi = pack4_bf16(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
@@ -273,15 +235,12 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   __shared__ __align__(8) uint64_t accum_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ int last_flag;
   __shared__ float inv_s[AMPH_MAX_NODES];
 
   pdl_launch_dependents();                          // the consumer kernel may get resident and wait
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool fused = prm.epi.mode != TC_EPI_NONE;
-  // SWIGLU: consecutive blocks (one cluster) take the gate tile and the up tile of the same features
-  const int tile = prm.epi.mode == TC_EPI_SWIGLU ? (int)(blockIdx.x & 1) * prm.tiles_per_seg + (int)(blockIdx.x >> 1)
-                                                 : (int)blockIdx.x;
-  const int split = blockIdx.y;
+  const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
   const int row0 = (tile - seg * prm.tiles_per_seg) * kTileM;       // first weight row of this tile
   const int kb_lo = (int)((long long)split * prm.kblocks / prm.splits);
@@ -373,11 +332,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag) : false);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int feat = seg * prm.tiles_per_seg * kTileM + row0 + quarter * 32 + lane;
-    // plain mode: fp32 partial tile to global memory; fused mode: to this CTA's shared memory ([row][128], the
-    // operand ring is idle by now) for the cluster-wide reduction below
-    float* out = fused ? reinterpret_cast<float*>(smem) + quarter * 32 + lane
-                       : prm.P + (size_t)split * prm.split_stride + feat;
-    const size_t out_ld = fused ? (size_t)kTileM : (size_t)prm.ld;
+    float* out = prm.P + (size_t)split * prm.split_stride + feat;
     for (int c0 = 0; c0 < nt; c0 += 16) {
       if (c0 >= prm.rows) break;
       uint32_t v[16];
@@ -396,10 +351,23 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       }
 #pragma unroll
       for (int j = 0; j < 16; ++j)
-        if (c0 + j < prm.rows) out[(size_t)(c0 + j) * out_ld] = __uint_as_float(v[j]);
+        if (c0 + j < prm.rows) out[(size_t)(c0 + j) * prm.ld] = __uint_as_float(v[j]);
     }
-    if (fused) {
-      for (int r = threadIdx.x - 64; r < prm.rows; r += 128) {   // deferred RMS division of every row
+    if (prm.epi.mode != TC_EPI_NONE) {
+      // Last arriver at this tile (both tiles of a gate / up pair for SWIGLU) reduces and finishes it.
+      const int et = threadIdx.x - 64;
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et == 0) {
+        const bool pair = prm.epi.mode == TC_EPI_SWIGLU;
+        const int idx = pair ? tile % prm.tiles_per_seg : tile;
+        const int target = (pair ? 2 : 1) * prm.splits;
+        const int old = atomicAdd(&prm.epi.counters[idx], 1);
+        const int last = (old == target - 1) && !abort_flag;
+        if (old == target - 1) prm.epi.counters[idx] = 0;        // ready for the next launch
+        last_flag = last;
+      }
+      for (int r = et; r < prm.rows; r += 128) {
         float sc = 1.0f;
         if (prm.epi.rs.ss != nullptr) {
           float tot = 0.f;
@@ -408,18 +376,15 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         }
         inv_s[r] = sc;
       }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (last_flag) {
+        __threadfence();
+        fused_epilogue(prm, tile, et, inv_s);
+      }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (fused) {
-    // Every CTA of the cluster has staged its tile; each finishes its share of the rows, reading the peers'
-    // tiles through distributed shared memory.  No CTA may leave before its peers have read its tile.
-    cluster_sync_all();
-    if (warp >= 2)
-      fused_epilogue(prm, tile, threadIdx.x - 64, inv_s, smem_u32(smem), (int)cluster_rank(), (int)cluster_size());
-    cluster_sync_all();
-  }
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
@@ -487,8 +452,8 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
 bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out, int in, int rows, float* P,
                     size_t p_floats, int* splits_out, size_t* split_stride, cudaStream_t st, const TcEpilogue* epi) {
   if (!g || xb < 0 || xb >= g->n_x) return false;
-  const bool fused = epi && epi->mode != TC_EPI_NONE;
-  if (fused) {
+  if (epi && epi->mode != TC_EPI_NONE) {
+    if (!epi->counters || n_seg * (out / kTileM) > kTcCounterInts) return false;
     if (epi->mode == TC_EPI_RESIDUAL && n_seg != 1) return false;
     if (epi->mode == TC_EPI_SWIGLU && n_seg != 2) return false;
     if (epi->mode == TC_EPI_QKV_ROPE &&
@@ -504,14 +469,9 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   int splits = (2 * g->sm_count) / tiles;
   if (splits > kblocks / 4) splits = kblocks / 4;
   if (splits > 16) splits = 16;
-  if (fused) {
-    if (splits > 8) splits = 8;                           // the K splits of a tile form one cluster (at most 8 CTAs)
-    if (epi->mode == TC_EPI_SWIGLU) splits = 1;           // its cluster pairs the gate tile with the up tile
-  } else {
-    while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
-    if ((size_t)nt * ld > p_floats) return false;
-  }
+  while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
   if (splits < 1) splits = 1;
+  if ((size_t)nt * ld > p_floats) return false;
   TmapPack pack;
   memset(&pack, 0, sizeof pack);
   for (int s = 0; s < n_seg; ++s) {
@@ -546,14 +506,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.err_flag = g->err_flag;
   prm.epi = epi ? *epi : TcEpilogue();
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  if (fused) {
-    const bool pair = epi->mode == TC_EPI_SWIGLU;
-    const cudaError_t e = launch_pdl_cluster(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pair ? 2 : 1,
-                                             pair ? 1 : splits, pack, prm);
-    if (e != cudaSuccess) { cudaGetLastError(); return false; }
-  } else {
-    launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
-  }
+  launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
   *split_stride = prm.split_stride;
   return true;

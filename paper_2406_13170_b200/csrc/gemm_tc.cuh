@@ -10,17 +10,18 @@ namespace amph {
 
 struct TcGemm;
 
-// Work fused into the projection kernel.  The CTAs that hold the K splits of one 128-feature tile are launched
-// as a thread-block cluster; each stages its fp32 partial tile in shared memory, and after a cluster barrier
-// every CTA sums, in split order and through distributed shared memory, its share of the rows and applies:
+// Work fused into the projection kernel.  Every CTA still leaves its split-K partial tile in P; the CTA that
+// arrives last at a tile (a counter per tile, no waiting) sums the partials in split order and applies:
 //   QKV_ROPE : three segments q, k, v of width n_heads * head_dim: deferred RMS division, rotary embedding,
 //              q -> q buffer, k / v -> KV-cache slots of the row table;
 //   RESIDUAL : x += y; xn = gain * x (not normalised); ss_part[row][tile] = sum of squares over the tile;
 //   SWIGLU   : two segments gate, up: deferred RMS division, act = silu(gate) * up.
 enum { TC_EPI_NONE = 0, TC_EPI_QKV_ROPE = 1, TC_EPI_RESIDUAL = 2, TC_EPI_SWIGLU = 3 };
+constexpr int kTcCounterInts = 4096;
 
 struct TcEpilogue {
   int mode = TC_EPI_NONE;
+  int* counters = nullptr;        // kTcCounterInts ints, all zero between launches
   RowScale rs;                    // QKV_ROPE, SWIGLU: division left over from the norm that fed this projection
   float* x = nullptr;             // RESIDUAL: fp32 residual stream [rows][out]
   void* xn = nullptr;             //           bf16 gain * x
