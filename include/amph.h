@@ -52,8 +52,7 @@ enum { AMPH_DTYPE_F32 = 0, AMPH_DTYPE_BF16 = 1 };
 /* amph_config.flags */
 enum {
   AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
-  AMPH_FLAG_NO_GRAPH = 2,       /* launch kernels one by one instead of replaying a CUDA graph */
-  AMPH_FLAG_NO_FUSED_EPILOGUE = 4 /* keep rotary / residual / SwiGLU in kernels of their own (A/B check) */
+  AMPH_FLAG_NO_GRAPH = 2        /* launch kernels one by one instead of replaying a CUDA graph */
 };
 
 #define AMPH_MAX_HEADS_K 8

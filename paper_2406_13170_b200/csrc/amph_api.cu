@@ -40,7 +40,7 @@ struct Layout {
   size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
-  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b, tc_counters;
+  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
   size_t partial_floats;
   int attn_splits;
 };
@@ -228,9 +228,8 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.att_ml = l.take(4 * (size_t)splits * c.n_heads * Mcap * 2);
   l.logits = l.take(4 * (size_t)Mcap * V);
   l.d_logits = l.take(4 * (size_t)kMaxK * V);
-  l.ss_a = l.take(4 * (size_t)Mcap * 128);
-  l.ss_b = l.take(4 * (size_t)Mcap * 128);
-  l.tc_counters = l.take(sizeof(int) * kTcCounterInts);
+  l.ss_a = l.take(4 * (size_t)Mcap * 32);
+  l.ss_b = l.take(4 * (size_t)Mcap * 32);
   *L = l;
   *Mcap_out = Mcap;
   const size_t per_layer = 2 * (size_t)c.n_heads * c.max_ctx * c.head_dim * esz;
@@ -308,38 +307,21 @@ void* xbuf_ptr(amph_ctx* ctx, int xb) {
   return ctx->ws + off[xb];
 }
 
-PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows,
-                         TcEpilogue* epi, bool* fused);
+PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows);
 
-// epi / fused: work the tensor-core kernel may finish itself (see TcEpilogue); *fused tells whether it did.
-// When it did not (plain kernel, uncovered shape) the caller runs the separate kernel on the returned sums.
-PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows,
-                    TcEpilogue* epi = nullptr, bool* fused = nullptr) {
+PartialView project(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
   ProfScope ps(ctx, AMPH_PROF_PROJECTION);
   if (ps.rec) ctx->prof_bytes += (int64_t)n_seg * out * in * (int64_t)ctx->esz;
-  return project_impl(ctx, xb, w, n_seg, out, in, rows, epi, fused);
+  return project_impl(ctx, xb, w, n_seg, out, in, rows);
 }
 
-PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows,
-                         TcEpilogue* epi, bool* fused) {
+PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg, int out, int in, int rows) {
   float* P = ctx->at<float>(ctx->lay.partial);
   PartialView pv;
   ctx->last_proj_one_wave = false;
-  if (fused) *fused = false;
   if (ctx->tc) {
     int splits = 0;
     size_t stride = 0;
-    if (epi) epi->counters = ctx->at<int>(ctx->lay.tc_counters);
-    if (epi && fused && !(ctx->cfg.flags & AMPH_FLAG_NO_FUSED_EPILOGUE) &&
-        tc_gemm_launch(ctx->tc, xb, w, n_seg, out, in, rows, P, ctx->lay.partial_floats, &splits, &stride,
-                       ctx->stream, epi)) {
-      *fused = true;
-      pv.p = P;
-      pv.splits = splits;
-      pv.ld = n_seg * out;
-      pv.split_stride = stride;
-      return pv;
-    }
     if (tc_gemm_launch(ctx->tc, xb, w, n_seg, out, in, rows, P, ctx->lay.partial_floats, &splits, &stride,
                        ctx->stream)) {
       ctx->last_proj_one_wave = (long long)n_seg * (out / 128) * splits <= 2LL * ctx->sm_count;
@@ -360,41 +342,30 @@ PartialView project_impl(amph_ctx* ctx, int xb, const void* const* w, int n_seg,
   return pv;
 }
 
-RowScale row_scale_of(const amph_ctx* ctx, size_t off, int chunks) {
+RowScale row_scale_of(const amph_ctx* ctx, size_t off) {
   RowScale rs;
-  if (chunks <= 0) return rs;
   rs.ss = ctx->at<float>(off);
-  rs.chunks = chunks;
+  rs.chunks = (ctx->cfg.d_model + kScaleChunkCols - 1) / kScaleChunkCols;
   rs.d = ctx->cfg.d_model;
   rs.eps = ctx->cfg.rms_eps;
   return rs;
 }
 
 // One decoder layer over the rows described by `meta`.
-// Entry: xn holds the input of the q/k/v projections: attn_norm * x / rms(x) if entry_chunks == 0, else
-// attn_norm * x with the row sums of squares in ss_a as entry_chunks partial sums per row (the division is
-// applied after the projection).
-// Exit: x is updated.  With next_gain and no hid: xn = next_gain * x and ss_a holds the sums of squares; the
-// number of partial sums per row is returned.  With hid: xn and hid hold the normalised rows (returns 0).
-// Where the tensor-core kernel covers the shape, rotary / KV write, residual update and SwiGLU run inside
-// the projection kernels; otherwise the separate kernels run on the projection's partial sums.
-int layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
-                  int rows, int ctx_hi, const void* next_gain, float* hid, int entry_chunks) {
+// Entry: xn holds the input of the q/k/v projections: attn_norm * x / rms(x) if !entry_deferred, else
+// attn_norm * x with the row sums of squares in ss_a (the division is applied after the projection).
+// Exit: x is updated.  With next_gain and no hid: xn = next_gain * x, sums of squares in ss_a (deferred form
+// for the next layer; returns true).  With hid: xn and hid hold the normalised rows (returns false).
+bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
+                   int rows, int ctx_hi, const void* next_gain, float* hid, bool entry_deferred) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const int chunks_fused = c.d_model / 128, chunks_plain = (c.d_model + kScaleChunkCols - 1) / kScaleChunkCols;
-  bool fused = false;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
-  TcEpilogue eq;
-  eq.mode = TC_EPI_QKV_ROPE;
-  eq.rs = row_scale_of(ctx, l.ss_a, entry_chunks);
-  eq.meta = meta; eq.rope = rope; eq.q = ctx->ws + l.q; eq.kc = kv.k; eq.vc = kv.v;
-  eq.n_heads = c.n_heads; eq.head_dim = c.head_dim; eq.max_ctx = c.max_ctx;
-  PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows, &eq, &fused);
-  if (!fused) {
-    ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
-    launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st, eq.rs);
+  PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
+  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st,
+                  entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale());
   }
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
@@ -402,43 +373,26 @@ int layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Row
                         c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr);
   }
   const void* wo[1] = {w.wo};
-  TcEpilogue eo;
-  eo.mode = TC_EPI_RESIDUAL;
-  eo.x = x; eo.xn = ctx->ws + l.xn; eo.gain = w.ffn_norm; eo.ss_part = ctx->at<float>(l.ss_b);
-  P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows, &eo, &fused);
-  int chunks_b = chunks_fused;
-  if (!fused) {
-    ProfScope ps(ctx, AMPH_PROF_NORM);
-    launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st,
-                       ctx->last_proj_one_wave);
-    chunks_b = chunks_plain;
+  P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_NORM);
+  launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st,
+                     ctx->last_proj_one_wave);
   }
   const void* gu[2] = {w.w_gate, w.w_up};
-  TcEpilogue eg;
-  eg.mode = TC_EPI_SWIGLU;
-  eg.rs = row_scale_of(ctx, l.ss_b, chunks_b);
-  eg.act = ctx->ws + l.act;
-  P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows, &eg, &fused);
-  if (!fused) {
-    ProfScope ps(ctx, AMPH_PROF_SWIGLU);
-    launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, eg.rs, ctx->last_proj_one_wave);
+  P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
+  { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
+  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b), ctx->last_proj_one_wave);
   }
   const void* wd[1] = {w.w_down};
-  if (hid != nullptr) {
-    P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
-    ProfScope ps(ctx, AMPH_PROF_NORM);
-    launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, hid, c.rms_eps, rows, c.d_model, st);
-    return 0;
-  }
-  TcEpilogue ed;
-  ed.mode = TC_EPI_RESIDUAL;
-  ed.x = x; ed.xn = ctx->ws + l.xn; ed.gain = next_gain; ed.ss_part = ctx->at<float>(l.ss_a);
-  P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows, &ed, &fused);
-  if (fused) return next_gain ? chunks_fused : 0;
+  P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
   ProfScope ps(ctx, AMPH_PROF_NORM);
+  if (hid != nullptr) {
+    launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, hid, c.rms_eps, rows, c.d_model, st);
+    return false;
+  }
   launch_resid_scale(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_a), rows, c.d_model, st,
                      ctx->last_proj_one_wave && next_gain != nullptr);
-  return next_gain ? chunks_plain : 0;
+  return next_gain != nullptr;
 }
 
 // Target forward of the rows in `tok` under meta_v; leaves post-final-norm rows in hidden and xn.
@@ -460,7 +414,7 @@ void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
   launch_resid_norm(x, none, 0, 0, ctx->layers[0].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                     c.d_model, st);
   }
-  int deferred = 0;
+  bool deferred = false;
   for (int i = 0; i < c.n_layers; ++i) {
     const bool last = i + 1 == c.n_layers;
     deferred = layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
@@ -501,7 +455,7 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
     }
-    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr, 0);
+    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr, false);
     in_feat = hbuf;
   }
 }

@@ -47,7 +47,6 @@ struct TcParams {
   int stages;
   int l2_prefetch;          // weight tiles (beyond the ring) each CTA pulls into L2 before it waits
   int* err_flag;
-  TcEpilogue epi;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -130,103 +129,6 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ float4 sum_tile4(const TcParams& prm, int r, int col) {
-  const float* p = prm.P + (size_t)r * prm.ld + col;
-  float4 acc = __ldcg(reinterpret_cast<const float4*>(p));
-  for (int s = 1; s < prm.splits; ++s) {                         // split order: deterministic
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(p + (size_t)s * prm.split_stride));
-    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-  }
-  return acc;
-}
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
-  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  uint2 u;
-  u.x = *reinterpret_cast<const unsigned*>(&lo);
-  u.y = *reinterpret_cast<const unsigned*>(&hi);
-  return u;
-}
-__device__ __forceinline__ float4 unpack4_bf16(const __nv_bfloat16* p) {
-  const uint2 u = *reinterpret_cast<const uint2*>(p);
-  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-                     __uint_as_float(u.y & 0xffff0000u));
-}
-
-// Runs in the CTA that completed a tile: et = 0..127 indexes the four epilogue warps' threads,
-// inv_s[r] is the deferred RMS division of row r (1 when none).
-__device__ void fused_epilogue(const TcParams& prm, int tile, int et, const float* inv_s) {
-  const TcEpilogue& e = prm.epi;
-  typedef __nv_bfloat16 bf16;
-  const int rows = prm.rows, tps = prm.tiles_per_seg;
-  const int lane = et & 31, ew = et >> 5;
-  if (e.mode == TC_EPI_RESIDUAL) {
-    const int d = prm.ld, c = tile * kTileM + 4 * lane;
-    for (int r = ew; r < rows; r += 4) {
-      float4 v = sum_tile4(prm, r, c);
-      float* xr = e.x + (size_t)r * d + c;
-      const float4 o = *reinterpret_cast<const float4*>(xr);
-      v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-      *reinterpret_cast<float4*>(xr) = v;
-      if (e.gain != nullptr) {
-        const float4 g = unpack4_bf16(reinterpret_cast<const bf16*>(e.gain) + c);
-        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.xn) + (size_t)r * d + c) =
-            pack4_bf16(g.x * v.x, g.y * v.y, g.z * v.z, g.w * v.w);
-        float ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        for (int o2 = 16; o2 > 0; o2 >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o2);
-        if (lane == 0) e.ss_part[(size_t)r * tps + tile] = ss;
-      }
-    }
-  } else if (e.mode == TC_EPI_SWIGLU) {
-    const int f = prm.ld / 2, c = (tile % tps) * kTileM + 4 * lane;
-    for (int r = ew; r < rows; r += 4) {
-      const float sc = inv_s[r];
-      const float4 g = sum_tile4(prm, r, c), u = sum_tile4(prm, r, f + c);
-      float t0 = g.x * sc, t1 = g.y * sc, t2 = g.z * sc, t3 = g.w * sc;
-      t0 = t0 / (1.0f + expf(-t0)) * (u.x * sc);
-      t1 = t1 / (1.0f + expf(-t1)) * (u.y * sc);
-      t2 = t2 / (1.0f + expf(-t2)) * (u.z * sc);
-      t3 = t3 / (1.0f + expf(-t3)) * (u.w * sc);
-      *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.act) + (size_t)r * f + c) = pack4_bf16(t0, t1, t2, t3);
-    }
-  } else if (e.mode == TC_EPI_QKV_ROPE) {
-    const int dh = e.head_dim, half = dh >> 1, quads = half >> 2, d = e.n_heads * dh;
-    const int seg = tile / tps, feat0 = (tile - seg * tps) * kTileM;
-    const int item = et & 15, rsub = et >> 4;                  // 16 items (4 rotation pairs each) per row
-    const int hh = item / quads, i = (item - hh * quads) * 4;
-    const int c0 = feat0 + hh * dh + i, c1 = c0 + half;
-    const int h = c0 / dh;
-    const int n_rows = e.meta->n_rows;
-    for (int r = rsub; r < rows; r += 8) {
-      const float sc = inv_s[r];
-      float4 a = sum_tile4(prm, r, seg * d + c0), b = sum_tile4(prm, r, seg * d + c1);
-      a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
-      const int slot = e.meta->slot[r];
-      const bool store = r < n_rows && slot >= 0 && slot < e.max_ctx;
-      const size_t co = ((size_t)h * e.max_ctx + (store ? slot : 0)) * dh + i;
-      if (seg == 2) {
-        if (store) {
-          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.vc) + co) = pack4_bf16(a.x, a.y, a.z, a.w);
-          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.vc) + co + half) = pack4_bf16(b.x, b.y, b.z, b.w);
-        }
-        continue;
-      }
-      const float4 cs0 = *reinterpret_cast<const float4*>(e.rope + r * half + i);
-      const float4 cs1 = *reinterpret_cast<const float4*>(e.rope + r * half + i + 2);
-      const uint2 lo = pack4_bf16(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
-                                  a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w);
-      const uint2 hi = pack4_bf16(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
-                                  b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w);
-      if (seg == 0) {
-        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.q) + (size_t)r * d + c0) = lo;
-        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.q) + (size_t)r * d + c1) = hi;
-      } else if (store) {
-        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.kc) + co) = lo;
-        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(e.kc) + co + half) = hi;
-      }
-    }
-  }
-}
-
 __global__ void __launch_bounds__(kThreads)
 tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -235,8 +137,6 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   __shared__ __align__(8) uint64_t accum_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ int last_flag;
-  __shared__ float inv_s[AMPH_MAX_NODES];
 
   pdl_launch_dependents();                          // the consumer kernel may get resident and wait
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -353,35 +253,6 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       for (int j = 0; j < 16; ++j)
         if (c0 + j < prm.rows) out[(size_t)(c0 + j) * prm.ld] = __uint_as_float(v[j]);
     }
-    if (prm.epi.mode != TC_EPI_NONE) {
-      // Last arriver at this tile (both tiles of a gate / up pair for SWIGLU) reduces and finishes it.
-      const int et = threadIdx.x - 64;
-      __threadfence();
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (et == 0) {
-        const bool pair = prm.epi.mode == TC_EPI_SWIGLU;
-        const int idx = pair ? tile % prm.tiles_per_seg : tile;
-        const int target = (pair ? 2 : 1) * prm.splits;
-        const int old = atomicAdd(&prm.epi.counters[idx], 1);
-        const int last = (old == target - 1) && !abort_flag;
-        if (old == target - 1) prm.epi.counters[idx] = 0;        // ready for the next launch
-        last_flag = last;
-      }
-      for (int r = et; r < prm.rows; r += 128) {
-        float sc = 1.0f;
-        if (prm.epi.rs.ss != nullptr) {
-          float tot = 0.f;
-          for (int c = 0; c < prm.epi.rs.chunks; ++c) tot += prm.epi.rs.ss[r * prm.epi.rs.chunks + c];
-          sc = 1.0f / sqrtf(tot / (float)prm.epi.rs.d + prm.epi.rs.eps);
-        }
-        inv_s[r] = sc;
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (last_flag) {
-        __threadfence();
-        fused_epilogue(prm, tile, et, inv_s);
-      }
-    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -450,15 +321,8 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
 }
 
 bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out, int in, int rows, float* P,
-                    size_t p_floats, int* splits_out, size_t* split_stride, cudaStream_t st, const TcEpilogue* epi) {
+                    size_t p_floats, int* splits_out, size_t* split_stride, cudaStream_t st) {
   if (!g || xb < 0 || xb >= g->n_x) return false;
-  if (epi && epi->mode != TC_EPI_NONE) {
-    if (!epi->counters || n_seg * (out / kTileM) > kTcCounterInts) return false;
-    if (epi->mode == TC_EPI_RESIDUAL && n_seg != 1) return false;
-    if (epi->mode == TC_EPI_SWIGLU && n_seg != 2) return false;
-    if (epi->mode == TC_EPI_QKV_ROPE &&
-        (n_seg != 3 || epi->head_dim < 8 || kTileM % epi->head_dim || out != epi->n_heads * epi->head_dim)) return false;
-  }
   if (out % kTileM || in % kTileK || n_seg < 1 || n_seg > kMaxSeg || rows < 1) return false;
   if (g->xcols[xb] != in) return false;
   const int nt = rows <= 16 ? 16 : (rows + 15) / 16 * 16;
@@ -504,7 +368,6 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
     prm.l2_prefetch = (int)(pf > 32 ? 32 : pf);
   }
   prm.err_flag = g->err_flag;
-  prm.epi = epi ? *epi : TcEpilogue();
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
