@@ -28,6 +28,19 @@ __device__ __forceinline__ float sum_partials(const PartialView& P, int row, int
   return acc;
 }
 
+// The partial sums sit in L2, one round trip each: the loads of a batch of N splits are issued together,
+// then added in split order.
+template <int N>
+__device__ __forceinline__ void add_splits(const float* p, size_t stride, int s0, int splits, float4& acc) {
+  float4 v[N];
+#pragma unroll
+  for (int s = 0; s < N; ++s)
+    if (s0 + s < splits) v[s] = *reinterpret_cast<const float4*>(p + (size_t)(s0 + s) * stride);
+#pragma unroll
+  for (int s = 0; s < N; ++s)
+    if (s0 + s < splits) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
+}
+
 __device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, int col) {
   const float* p = P.p + (size_t)row * P.ld + col;
   float4 acc = *reinterpret_cast<const float4*>(p);
@@ -36,6 +49,15 @@ __device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, i
     const float4 v = *reinterpret_cast<const float4*>(p + (size_t)s * P.split_stride);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
+  return acc;
+}
+// Same sum for kernels with registers to spare and many splits to read (the residual kernels).
+__device__ __forceinline__ float4 sum_partials4_wide(const PartialView& P, int row, int col) {
+  const float* p = P.p + (size_t)row * P.ld + col;
+  float4 acc = *reinterpret_cast<const float4*>(p);
+  const int n = P.splits;
+  if (n == 1) return acc;
+  for (int s0 = 1; s0 < n; s0 += 8) add_splits<8>(p, P.split_stride, s0, n, acc);
   return acc;
 }
 
@@ -57,6 +79,7 @@ __device__ __forceinline__ float4 load4(const bf16* p) {
 __device__ __forceinline__ float row_scale(const RowScale& rs, int row) {
   if (rs.ss == nullptr) return 1.0f;
   float tot = 0.f;
+#pragma unroll 8
   for (int c = 0; c < rs.chunks; ++c) tot += rs.ss[row * rs.chunks + c];       // fixed order
   return 1.0f / sqrtf(tot / (float)rs.d + rs.eps);
 }
@@ -162,7 +185,7 @@ resid_scale_kernel(float* __restrict__ x, PartialView P, int col_off, int mode, 
   float ss = 0.f;
   if (c < d) {
     float* xr = x + (size_t)r * d + c;
-    float4 v = sum_partials4(P, r, col_off + c);
+    float4 v = sum_partials4_wide(P, r, col_off + c);
     if (mode == 1) { const float4 o = load4(xr); v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
     store4(xr, v);
     if (gain != nullptr) {
@@ -399,21 +422,45 @@ __global__ void attn_combine_kernel(const float* __restrict__ po, const float* _
   pdl_wait();
   if (!early) pdl_launch_dependents();
   const int r = blockIdx.x, h = blockIdx.y;
+  const size_t stride = (size_t)n_heads * rows_cap, o0 = (size_t)h * rows_cap + r;
+  if (splits <= 16) {
+    // every load of the launch is issued before the first use: (max, sum) of all splits, then the partial
+    // outputs of all splits for this thread's column
+    float2 ml[16];
+#pragma unroll
+    for (int s = 0; s < 16; ++s)
+      ml[s] = s < splits ? *reinterpret_cast<const float2*>(pml + (o0 + s * stride) * 2) : make_float2(-INFINITY, 0.f);
+    for (int c = threadIdx.x; c < dh; c += blockDim.x) {
+      float v[16];
+#pragma unroll
+      for (int s = 0; s < 16; ++s) v[s] = s < splits ? po[(o0 + s * stride) * dh + c] : 0.f;
+      float M = -INFINITY;
+#pragma unroll
+      for (int s = 0; s < 16; ++s) M = fmaxf(M, ml[s].x);
+      float den = 0.f, num = 0.f;
+#pragma unroll
+      for (int s = 0; s < 16; ++s)
+        if (ml[s].x != -INFINITY) {
+          const float w = expf(ml[s].x - M);
+          den += ml[s].y * w;
+          num += v[s] * w;
+        }
+      out[(size_t)r * n_heads * dh + h * dh + c] = from_f<T>(den > 0.f ? num / den : 0.f);
+    }
+    return;
+  }
   float M = -INFINITY;
-  for (int s = 0; s < splits; ++s)
-    M = fmaxf(M, pml[(((size_t)s * n_heads + h) * rows_cap + r) * 2]);
+  for (int s = 0; s < splits; ++s) M = fmaxf(M, pml[(o0 + s * stride) * 2]);
   float den = 0.f;
   for (int s = 0; s < splits; ++s) {
-    const size_t o = ((size_t)s * n_heads + h) * rows_cap + r;
-    const float m = pml[o * 2];
-    if (m != -INFINITY) den += pml[o * 2 + 1] * expf(m - M);
+    const float m = pml[(o0 + s * stride) * 2];
+    if (m != -INFINITY) den += pml[(o0 + s * stride) * 2 + 1] * expf(m - M);
   }
   for (int c = threadIdx.x; c < dh; c += blockDim.x) {
     float num = 0.f;
     for (int s = 0; s < splits; ++s) {
-      const size_t o = ((size_t)s * n_heads + h) * rows_cap + r;
-      const float m = pml[o * 2];
-      if (m != -INFINITY) num += po[o * dh + c] * expf(m - M);
+      const float m = pml[(o0 + s * stride) * 2];
+      if (m != -INFINITY) num += po[(o0 + s * stride) * dh + c] * expf(m - M);
     }
     out[(size_t)r * n_heads * dh + h * dh + c] = from_f<T>(den > 0.f ? num / den : 0.f);
   }
