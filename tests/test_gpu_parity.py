@@ -85,3 +85,21 @@ def test_long_prompt_many_attention_splits_bf16():
                      kv_check_layers=(0, 1, 2))
     print(rep)
     model.close()
+
+
+@pytest.mark.parametrize("variant", [dict(n_sal=1), dict(aeb_layers=2), dict(n_sal=1, aeb_layers=2)],
+                         ids=["one-sal", "alpha-two-aeb-layers", "one-sal-two-aeb-layers"])
+@pytest.mark.parametrize("base", ["tiny", "small_bf16"])
+def test_draft_module_variants(base, variant):
+    """The draft-module variants the paper evaluates: a single adaptation layer (the "One-Adaptation-Layer"
+    ablation of Section 4.5: every head then reads h1) and the two-layer Auto-embedding Block ("Amphista-alpha",
+    Appendix A.2.3)."""
+    shape = inputs.get_shape(base).with_(**variant)
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    model, orc = _setup(shape, topo)
+    prompt = inputs.make_prompt(shape).tolist()
+    bf = shape.dtype == "bf16"
+    rep = run_parity(model, orc, shape, topo, prompt, 4, TOL_BF16 if bf else TOL_F32, TIE_BF16 if bf else TIE_F32, True)
+    print(rep)
+    assert rep.steps == 4 and max(rep.accepted) >= 3
+    model.close()

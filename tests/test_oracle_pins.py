@@ -412,3 +412,70 @@ def test_storage_rounding_mode_is_identity_without_rounding_and_small_with_bf16(
     for a, c in zip(outs[0], outs[2]):
         err = float((a - c).abs().max()) / max(1.0, float(a.abs().max()))
         assert 0.0 < err < 3e-2
+
+
+# --------------------------------------------------------------------------------------
+# draft-module variants (Section 4.5 "One-Adaptation-Layer", Appendix A.2.3 "Amphista-alpha")
+# --------------------------------------------------------------------------------------
+def test_variant_one_adaptation_layer_feeds_every_head_from_stage_one():
+    """With a single adaptation layer every head reads h1 (Section 4.5): the variant's stage-1 output
+    equals the two-stage model's (same weights, same inputs), and each head row is the Eq. 2 form of it."""
+    two = _oracle(MICRO, std=0.2)
+    one_shape = MICRO.with_(n_sal=1)
+    one = ao.Oracle(one_shape, inputs.make_weights(MICRO, seed=0, std=0.2), dtype=torch.float64)
+    prompt = inputs.make_prompt(MICRO).tolist()
+    t2, t1 = {}, {}
+    two.draft(two.prefill(prompt), t2)
+    st = one.prefill(prompt)
+    one.draft(st, t1)
+    assert len(st.sal_kv) == 1
+    assert torch.allclose(t1["h1"], t2["h1"], atol=1e-12)
+    base = t1["Hp"] - one.W("draft.pe")
+    for k in range(MICRO.K):
+        w, b = one.W(f"draft.mlp.{k}.w"), one.W(f"draft.mlp.{k}.b")
+        assert torch.allclose(base[k], t1["h1"] + torch.nn.functional.silu(w @ t1["h1"] + b), atol=1e-12)
+    # heads of the second half differ from the two-stage model (there they read h2), the first half does not
+    b2 = t2["Hp"] - two.W("draft.pe")
+    assert torch.allclose(base[: MICRO.K // 2], b2[: MICRO.K // 2], atol=1e-12)
+    assert not torch.allclose(base[MICRO.K // 2:], b2[MICRO.K // 2:], atol=1e-6)
+
+
+def test_variant_two_aeb_layers_is_composition_and_reduces_to_one():
+    """Amphista-alpha stacks two self-attention layers (Appendix A.2.3): the block is the composition of the
+    two layers, stays permutation equivariant, and with a zero output projection in the second layer the
+    residual makes it equal to the one-layer block."""
+    shape = MICRO.with_(aeb_layers=2)
+    w = inputs.make_weights(shape, seed=0, std=0.2)
+    orc = ao.Oracle(shape, w, dtype=torch.float64)
+    prompt = inputs.make_prompt(shape).tolist()
+    taps = {}
+    orc.draft(orc.prefill(prompt), taps)
+    assert torch.allclose(taps["attn_o"], orc.aeb(orc.aeb(taps["Hp"], 0), 1), atol=1e-12)
+    assert not torch.allclose(taps["attn_o"], orc.aeb(taps["Hp"], 0), atol=1e-6)
+    Hp = inputs.normal_tensor((shape.K, shape.d_model), 1.0, 9, "Hp", dtype=torch.float64)
+    two = lambda X: orc.aeb(orc.aeb(X, 0), 1)
+    p = [2, 0, 3, 1]
+    assert torch.allclose(two(Hp[p]), two(Hp)[p], atol=1e-10)
+    w0 = dict(w)
+    w0["draft.aeb.1.wo"] = torch.zeros_like(w["draft.aeb.1.wo"])
+    orc0 = ao.Oracle(shape, w0, dtype=torch.float64)
+    t0 = {}
+    orc0.draft(orc0.prefill(prompt), t0)
+    assert torch.allclose(t0["attn_o"], orc0.aeb(t0["Hp"], 0), atol=1e-12)
+
+
+@pytest.mark.parametrize("variant", [dict(n_sal=1), dict(aeb_layers=2)], ids=["one-sal", "two-aeb-layers"])
+def test_variants_stay_lossless(variant):
+    shape = MICRO.with_(**variant)
+    orc = ao.Oracle(shape, inputs.make_weights(shape, seed=0, std=0.2), dtype=torch.float64)
+    prompt = inputs.make_prompt(shape).tolist()
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    t = _tables(topo)
+    ref = orc.greedy_ar(prompt, 4 * (shape.K + 1) + 1)
+    st = orc.prefill(prompt)
+    out = []
+    for i in range(4):
+        leaf = t.leaves[i % len(t.leaves)]
+        emitted = orc.step(st, t, _plant(t, st.root, ref[len(out) + 1: len(out) + 1 + t.depth[leaf]], leaf), {})
+        out += emitted
+    assert out == ref[: len(out)] and st.root == ref[len(out)]
