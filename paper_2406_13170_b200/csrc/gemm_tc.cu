@@ -26,6 +26,7 @@ namespace {
 constexpr int kTileM = 128;           // weight rows per CTA (UMMA M)
 constexpr int kTileK = 64;            // bf16 elements per 128-byte swizzle row
 constexpr int kUmmaK = 16;            // K per tcgen05.mma for 16-bit inputs
+constexpr int kStageKb = 2;           // 64-wide K blocks fetched by one TMA copy (one pipeline stage)
 constexpr int kMaxSeg = 8;
 constexpr int kThreads = 192;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // a barrier wait gives up after one second
@@ -89,15 +90,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
-// Asks the TMA unit to bring one weight tile into L2 (no shared-memory destination, no barrier).
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+// The operands are described to the TMA unit as 3-D tensors (64 columns, rows, K block): one copy brings
+// kStageKb consecutive K blocks of a row range, each landing as its own 128-byte-swizzled K-major tile.
+// An SM retires roughly one tiled copy per 400 clocks whatever its size (measured with copies of 8 to
+// 32 KB), so larger copies are what lets L2-resident weights arrive faster than HBM delivers them.
+// The first coordinate is always 0 (16-byte rule); K blocks past the end of the tensor read as zeros.
+// Asks the TMA unit to bring the weight tiles of one stage into L2 (no shared-memory destination, no barrier).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int row, int kb) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(0), "r"(row), "r"(kb) : "memory");
 }
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(smem_u32(bar))
       : "memory");
 }
 
@@ -143,11 +149,16 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
   const int row0 = (tile - seg * prm.tiles_per_seg) * kTileM;       // first weight row of this tile
-  const int kb_lo = (int)((long long)split * prm.kblocks / prm.splits);
-  const int kb_hi = (int)((long long)(split + 1) * prm.kblocks / prm.splits);
+  // K range of this split in whole stages (kStageKb blocks), so that every copy starts on a stage boundary
+  const int units = (prm.kblocks + kStageKb - 1) / kStageKb;
+  const int kb_lo = (int)((long long)split * units / prm.splits) * kStageKb;
+  int kb_hi = (int)((long long)(split + 1) * units / prm.splits) * kStageKb;
+  if (kb_hi > prm.kblocks) kb_hi = prm.kblocks;
   const int nkb = kb_hi - kb_lo;
+  const int nit = (nkb + kStageKb - 1) / kStageKb;                  // pipeline iterations
   const int nt = prm.nt, stages = prm.stages;
-  const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
+  const uint32_t a_tile = kTileM * kTileK * 2, b_tile = (uint32_t)nt * kTileK * 2;     // one K block of each operand
+  const uint32_t a_bytes = kStageKb * a_tile, b_bytes = kStageKb * b_tile;
   const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint32_t tmem_cols = 32;
@@ -176,25 +187,25 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x) : "memory");
       // Weights do not depend on the previous kernel: fill the ring with weight tiles first, then wait for
       // the producer of the activations, then fetch the activation tiles of those stages.
-      const int npre = nkb < stages ? nkb : stages;
+      const int npre = nit < stages ? nit : stages;
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
-        tma_load_2d(smem + (size_t)i * stage_bytes, wmap, (kb_lo + i) * kTileK, row0, &full_bar[i]);
+        tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * kStageKb, &full_bar[i]);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
-      const int npf = nkb < npre + prm.l2_prefetch ? nkb : npre + prm.l2_prefetch;
-      for (int i = npre; i < npf; ++i) tma_prefetch_l2_2d(wmap, (kb_lo + i) * kTileK, row0);
+      const int npf = nit < npre + prm.l2_prefetch ? nit : npre + prm.l2_prefetch;
+      for (int i = npre; i < npf; ++i) tma_prefetch_l2_3d(wmap, row0, kb_lo + i * kStageKb);
       pdl_wait();
       for (int i = 0; i < npre; ++i)
-        tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, (kb_lo + i) * kTileK, 0, &full_bar[i]);
+        tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[i]);
       int issued = npre;
-      for (int i = npre; i < nkb; ++i) {
+      for (int i = npre; i < nit; ++i) {
         const int s = i % stages, round = i / stages;
         if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag)) break;
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        tma_load_2d(a, wmap, (kb_lo + i) * kTileK, row0, &full_bar[s]);
-        tma_load_2d(a + a_bytes, &maps.x, (kb_lo + i) * kTileK, 0, &full_bar[s]);
+        tma_load_3d(a, wmap, row0, kb_lo + i * kStageKb, &full_bar[s]);
+        tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[s]);
         issued = i + 1;
       }
       if (abort_flag) {                              // drain: let every copy this thread issued land
@@ -211,16 +222,19 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(nt);
       bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
+      for (int i = 0; i < nit && ok; ++i) {
         const int s = i % stages, round = i / stages;
         ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t adesc = umma_desc(a_addr), bdesc = umma_desc(a_addr + a_bytes);
+        const int nk = nkb - i * kStageKb < kStageKb ? nkb - i * kStageKb : kStageKb;   // blocks of the stage inside the K range
+        for (int kk = 0; kk < nk; ++kk) {
+          const uint64_t adesc = umma_desc(a_addr + (uint32_t)kk * a_tile), bdesc = umma_desc(a_addr + a_bytes + (uint32_t)kk * b_tile);
 #pragma unroll
-        for (int k = 0; k < kTileK / kUmmaK; ++k)      // +32 bytes (2 x 16 B) per K step inside the swizzle row
-          umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | k) ? 1u : 0u);
+          for (int k = 0; k < kTileK / kUmmaK; ++k)    // +32 bytes (2 x 16 B) per K step inside the swizzle row
+            umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+        }
         umma_commit(&empty_bar[s]);                    // frees the stage once these MMAs have read it
       }
       if (ok) umma_commit(&accum_bar);
@@ -284,11 +298,12 @@ struct TcGemm {
     auto it = cache.find(key);
     if (it != cache.end()) return &it->second;
     CUtensorMap m;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+    // (column within a K block, row, K block): stride of a row = its pitch, of a K block = 128 bytes
+    const cuuint64_t dims[3] = {(cuuint64_t)kTileK, (cuuint64_t)rows, (cuuint64_t)cols / kTileK};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)kTileK * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows, (cuuint32_t)kStageKb};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return nullptr;
@@ -332,6 +347,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   // K-splits: fill about two CTAs per SM, keep at least four 64-wide K blocks per CTA
   int splits = (2 * g->sm_count) / tiles;
   if (splits > kblocks / 4) splits = kblocks / 4;
+  if (splits > (kblocks + kStageKb - 1) / kStageKb) splits = (kblocks + kStageKb - 1) / kStageKb;
   if (splits > 16) splits = 16;
   while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
   if (splits < 1) splits = 1;
@@ -347,8 +363,8 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt);
   if (!mx) return false;
   pack.x = *mx;
-  const uint32_t stage_bytes = kTileM * kTileK * 2 + (((uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
-  int stages = (int)((100 * 1024) / stage_bytes);          // <= ~100 KB per CTA: two CTAs per SM
+  const uint32_t stage_bytes = kStageKb * kTileM * kTileK * 2 + ((kStageKb * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  int stages = (int)((110 * 1024) / stage_bytes);          // <= ~110 KB per CTA: two CTAs per SM
   if (stages > 8) stages = 8;
   if (stages < 2) stages = 2;
   TcParams prm;
@@ -364,7 +380,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   // about 40 MB of L2 for prefetched weight tiles, shared by the CTAs that can be resident at once
   {
     const long long resident = (long long)tiles * splits < 2LL * g->sm_count ? (long long)tiles * splits : 2LL * g->sm_count;
-    long long pf = (40LL << 20) / (resident * (kTileM * kTileK * 2));
+    long long pf = (40LL << 20) / (resident * (kStageKb * kTileM * kTileK * 2));
     prm.l2_prefetch = (int)(pf > 32 ? 32 : pf);
   }
   prm.err_flag = g->err_flag;
