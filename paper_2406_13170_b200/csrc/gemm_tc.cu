@@ -90,6 +90,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// One lane of a converged warp.  TMA and MMA instructions are issued by the elected lane while the other
+// lanes stay with it: issued by a lone thread of a diverged warp, a tcgen05.mma costs about 210 clocks
+// instead of the 48 that a 128 x 64 x 16 MMA occupies the tensor pipe (both measured), which would cap
+// a CTA at about 37 GB/s of weights.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t e;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+  return e != 0;
+}
+
 // The operands are described to the TMA unit as 3-D tensors (64 columns, rows, K block): one copy brings
 // kStageKb consecutive K blocks of a row range, each landing as its own 128-byte-swizzled K-major tile.
 // An SM retires roughly one tiled copy per 400 clocks whatever its size (measured with copies of 8 to
@@ -180,53 +190,63 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const uint32_t tmem_d = tmem_base_slot;
 
   if (warp == 0) {
-    // ---------------- TMA producer
-    if (lane == 0) {
-      const CUtensorMap* wmap = &maps.w[seg];
+    // ---------------- TMA producer (the warp stays converged, its elected lane issues)
+    const bool leader = elect_one();
+    const CUtensorMap* wmap = &maps.w[seg];
+    if (leader) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(wmap) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x) : "memory");
-      // Weights do not depend on the previous kernel: fill the ring with weight tiles first, then wait for
-      // the producer of the activations, then fetch the activation tiles of those stages.
-      const int npre = nit < stages ? nit : stages;
+    }
+    // Weights do not depend on the previous kernel: fill the ring with weight tiles first, then wait for
+    // the producer of the activations, then fetch the activation tiles of those stages.
+    const int npre = nit < stages ? nit : stages;
+    const int npf = nit < npre + prm.l2_prefetch ? nit : npre + prm.l2_prefetch;
+    if (leader) {
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
         tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * kStageKb, &full_bar[i]);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
-      const int npf = nit < npre + prm.l2_prefetch ? nit : npre + prm.l2_prefetch;
       for (int i = npre; i < npf; ++i) tma_prefetch_l2_3d(wmap, row0, kb_lo + i * kStageKb);
-      pdl_wait();
+    }
+    __syncwarp();
+    pdl_wait();
+    if (leader)
       for (int i = 0; i < npre; ++i)
         tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[i]);
-      int issued = npre;
-      for (int i = npre; i < nit; ++i) {
-        const int s = i % stages, round = i / stages;
-        if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag)) break;
+    __syncwarp();
+    int issued = npre;
+    for (int i = npre; i < nit; ++i) {
+      const int s = i % stages, round = i / stages;
+      if (!__all_sync(0xffffffffu, mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag))) break;
+      if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
         tma_load_3d(a, wmap, row0, kb_lo + i * kStageKb, &full_bar[s]);
         tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[s]);
-        issued = i + 1;
       }
-      if (abort_flag) {                              // drain: let every copy this thread issued land
-        const int first = issued > stages ? issued - stages : 0;
-        for (int i = first; i < issued; ++i) {
-          const int s = i % stages, round = i / stages;
-          const unsigned long long t0 = now_ns();
-          while (!mbar_try(&full_bar[s], round & 1) && now_ns() - t0 < kWaitLimitNs) {}
-        }
+      __syncwarp();
+      issued = i + 1;
+    }
+    if (abort_flag && lane == 0) {                     // drain: let every copy that was issued land
+      const int first = issued > stages ? issued - stages : 0;
+      for (int i = first; i < issued; ++i) {
+        const int s = i % stages, round = i / stages;
+        const unsigned long long t0 = now_ns();
+        while (!mbar_try(&full_bar[s], round & 1) && now_ns() - t0 < kWaitLimitNs) {}
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc(nt);
-      bool ok = true;
-      for (int i = 0; i < nit && ok; ++i) {
-        const int s = i % stages, round = i / stages;
-        ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
-        if (!ok) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // ---------------- MMA issuer (the warp stays converged, its elected lane issues)
+    const bool leader = elect_one();
+    const uint32_t idesc = umma_idesc(nt);
+    bool ok = true;
+    for (int i = 0; i < nit; ++i) {
+      const int s = i % stages, round = i / stages;
+      ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, &abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (leader) {
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
         const int nk = nkb - i * kStageKb < kStageKb ? nkb - i * kStageKb : kStageKb;   // blocks of the stage inside the K range
         for (int kk = 0; kk < nk; ++kk) {
@@ -237,8 +257,10 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         }
         umma_commit(&empty_bar[s]);                    // frees the stage once these MMAs have read it
       }
-      if (ok) umma_commit(&accum_bar);
+      __syncwarp();
     }
+    if (ok && leader) umma_commit(&accum_bar);
+    __syncwarp();
   } else {
     // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
     const int quarter = warp & 3;
