@@ -37,7 +37,7 @@ struct Layout {
     return off;
   }
   size_t state, tree, meta_v, meta_s, kv_tab, inv_freq, rope_v, rope_s;
-  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals;
+  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals, topk_cand;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
   size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
@@ -199,6 +199,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.next_tok = l.take(sizeof(int) * kMaxRows);
   l.topk_ids = l.take(sizeof(int) * kMaxK * kTopkStride);
   l.topk_vals = l.take(sizeof(float) * kMaxK * kTopkStride);
+  l.topk_cand = l.take(2 * sizeof(float) * kMaxK * kTopkCandChunks * kTopkStride);
   l.x = l.take(4 * Mcap * d);
   l.hidden = l.take(4 * Mcap * d);
   l.h1 = l.take(4 * Mcap * d);
@@ -511,7 +512,7 @@ amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
   P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                               // Eq. 6
   { ProfScope ps(ctx, AMPH_PROF_SELECT);
   launch_topk_heads(P, c.vocab, c.K, c.topk, ctx->at<int>(l.topk_ids), ctx->at<float>(l.topk_vals),
-                    ctx->at<float>(l.d_logits), st);
+                    ctx->at<float>(l.d_logits), ctx->at<float>(l.topk_cand), st);
   }
   { ProfScope ps(ctx, AMPH_PROF_OTHER);
   launch_tree_build(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.topk_ids), nullptr, ctx->at<int>(l.tok),

@@ -160,8 +160,10 @@ void launch_mlp_heads(PartialView P, const float* last, const void* const* bias,
 void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
                           cudaStream_t st);
 // per head k: top-c_k of row k of segment k; also stores the row into d_logits[k]
+// cand: scratch for the slices' candidates, kMaxK * kTopkCandChunks * kTopkStride (value, id) pairs
+constexpr int kTopkCandChunks = 32;
 void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids, float* vals,
-                       float* d_logits, cudaStream_t st);
+                       float* d_logits, float* cand, cudaStream_t st);
 void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st);
 
 // ---- control kernels

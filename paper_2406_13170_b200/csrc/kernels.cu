@@ -757,40 +757,74 @@ __device__ void block_best(float& v, int& i, float* sv, int* si) {
 
 struct TopkCounts { int c[kMaxK]; };
 
-__global__ void topk_heads_kernel(PartialView P, int vocab, TopkCounts ck, int* __restrict__ ids,
-                                  float* __restrict__ vals, float* __restrict__ d_logits, int mode) {
+// Stage 1: block (head k, chunk j) reduces the split-K partials of its slice of the head's logits, stores
+// them (debug tap) and selects the slice's own top-c_k in the order above.  Stage 2: one block per head
+// merges the slices' candidates.  The global top-c_k are each among their slice's top-c_k, so the result is
+// the exact top-c_k of the row, in order.
+constexpr int kTopkChunks = kTopkCandChunks;
+constexpr int kTopkThreads = 256;
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_slice_kernel(PartialView P, int vocab, int chunk, TopkCounts ck, float2* __restrict__ cand,
+                  float* __restrict__ d_logits, int vec) {
   pdl_wait();
   pdl_launch_dependents();
-  extern __shared__ __align__(16) float rowbuf[];       // the head's logits when they fit, else the global copy is used
+  extern __shared__ __align__(16) float slice[];
   __shared__ float sv[32];
   __shared__ int si[32];
-  const int k = blockIdx.x;
-  const int in_smem = mode & 1, vec = mode & 2;          // bit 0: row cached in shared memory; bit 1: 16-byte loads are aligned
+  const int k = blockIdx.x, j = blockIdx.y;
+  const int lo = j * chunk, hi = lo + chunk < vocab ? lo + chunk : vocab;
   float* grow = d_logits + (size_t)k * vocab;
-  for (int c = threadIdx.x * 4; c < vocab; c += blockDim.x * 4) {
-    if (vec && c + 3 < vocab) {
+  for (int c = lo + threadIdx.x * 4; c < hi; c += blockDim.x * 4) {
+    if (vec && c + 3 < hi) {
       const float4 v = sum_partials4(P, k, k * vocab + c);
       store4(grow + c, v);
-      if (in_smem) store4(rowbuf + c, v);
+      store4(slice + (c - lo), v);
     } else {
-      for (int e = c; e < vocab && e < c + 4; ++e) {
+      for (int e = c; e < hi && e < c + 4; ++e) {
         const float v = sum_partials(P, k, k * vocab + e);
         grow[e] = v;
-        if (in_smem) rowbuf[e] = v;
+        slice[e - lo] = v;
       }
     }
   }
   __syncthreads();
-  const float* row = in_smem ? rowbuf : grow;
   float pv = INFINITY;
   int pi = -1;
   for (int t = 0; t < ck.c[k]; ++t) {
     float bv = -INFINITY;
     int bi = 0x7fffffff;
-    for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
-      const float v = row[c];
-      const bool after_prev = v < pv || (v == pv && c > pi);     // strictly after the previous pick
+    for (int c = lo + threadIdx.x; c < hi; c += blockDim.x) {
+      const float v = slice[c - lo];
+      const bool after_prev = v < pv || (v == pv && c > pi);       // strictly after the previous pick
       if (after_prev && better(v, c, bv, bi)) { bv = v; bi = c; }
+    }
+    block_best(bv, bi, sv, si);
+    if (threadIdx.x == 0) cand[((size_t)k * gridDim.y + j) * kTopkStride + t] = make_float2(bv, __int_as_float(bi));
+    pv = bv; pi = bi;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_merge_kernel(const float2* __restrict__ cand, int n_chunks, TopkCounts ck, int* __restrict__ ids,
+                  float* __restrict__ vals) {
+  pdl_wait();
+  pdl_launch_dependents();
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  const int k = blockIdx.x, ckk = ck.c[k];
+  const int n = n_chunks * ckk;                                    // candidates of this head
+  float pv = INFINITY;
+  int pi = -1;
+  for (int t = 0; t < ckk; ++t) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int c = threadIdx.x; c < n; c += blockDim.x) {
+      const float2 e = cand[((size_t)k * n_chunks + c / ckk) * kTopkStride + c % ckk];
+      const int id = __float_as_int(e.y);
+      const bool after_prev = e.x < pv || (e.x == pv && id > pi);
+      if (id != 0x7fffffff && after_prev && better(e.x, id, bv, bi)) { bv = e.x; bi = id; }
     }
     block_best(bv, bi, sv, si);
     if (threadIdx.x == 0) { ids[k * kTopkStride + t] = bi; vals[k * kTopkStride + t] = bv; }
@@ -800,15 +834,18 @@ __global__ void topk_heads_kernel(PartialView P, int vocab, TopkCounts ck, int* 
 }
 
 void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids, float* vals, float* d_logits,
-                       cudaStream_t st) {
+                       float* cand, cudaStream_t st) {
   TopkCounts c;
   for (int k = 0; k < kMaxK; ++k) c.c[k] = k < K ? ck[k] : 0;
-  const size_t bytes = (size_t)vocab * sizeof(float);
   const int vec = vocab % 4 == 0 && P.ld % 4 == 0;
-  const int in_smem = bytes <= 200 * 1024;
-  if (in_smem) cudaFuncSetAttribute(topk_heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  launch_pdl(topk_heads_kernel, dim3(K), dim3(1024), in_smem ? bytes : 0, st, P, vocab, c, ids, vals, d_logits,
-             in_smem | (vec << 1));
+  int chunk = (vocab + kTopkChunks - 1) / kTopkChunks;
+  chunk = (chunk + 3) / 4 * 4;
+  const int n_chunks = (vocab + chunk - 1) / chunk;
+  const size_t bytes = (size_t)chunk * sizeof(float);
+  if (bytes > 48 * 1024) cudaFuncSetAttribute(topk_slice_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  launch_pdl(topk_slice_kernel, dim3(K, n_chunks), dim3(kTopkThreads), bytes, st, P, vocab, chunk, c,
+             reinterpret_cast<float2*>(cand), d_logits, vec);
+  launch_pdl(topk_merge_kernel, dim3(K), dim3(kTopkThreads), 0, st, reinterpret_cast<const float2*>(cand), n_chunks, c, ids, vals);
 }
 
 __global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ amax,
