@@ -80,6 +80,9 @@ typedef struct {
   int32_t aeb_layers;     /* 1 (the paper's design) or 2 (its "alpha" variant)              */
   int32_t topk[AMPH_MAX_HEADS_K]; /* candidates kept per head, each 1..AMPH_TOPK_STRIDE     */
   int32_t flags;          /* AMPH_FLAG_*                                                    */
+  int32_t lm_rank;        /* 0: each drafting head owns a [vocab, d] matrix (Eq. 6); r > 0: it owns two
+                           * low-rank factors a [r, d] and b [vocab, r], logits = b (a x) (Appendix A.2.4);
+                           * r a multiple of 8, r <= d_model                                  */
 } amph_config;
 
 /* Draft-tree topology (Appendix A.1): node 0 is the root (the token the target chose last);
@@ -123,7 +126,8 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
  *   w_gate, w_up [F,d], w_down [d,F]}; final_norm [d]; lm_head [V,d];
  *   draft.fc{s} [d,2d] (Eq. 1; input order [hidden ; token embedding]);
  *   draft.sal{s}.<the nine per-layer names>; draft.mlp.{k}.w [d,d], draft.mlp.{k}.b [d] (Eq. 2);
- *   draft.pe [K,d] (Eq. 4); draft.aeb.{l}.{wq,wk,wv,wo} [d,d] (Eq. 5); draft.lm_head.{k} [V,d] (Eq. 6).
+ *   draft.pe [K,d] (Eq. 4); draft.aeb.{l}.{wq,wk,wv,wo} [d,d] (Eq. 5); draft.lm_head.{k} [V,d] (Eq. 6),
+ *   or with lm_rank = r > 0: draft.lm_head.{k}.a [r,d] and draft.lm_head.{k}.b [V,r] (Appendix A.2.4).
  * May be called several times; AMPH_ERR_MISSING_WEIGHT is reported by amph_prefill if a tensor
  * was never given.  Pointers are borrowed. */
 amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t n);

@@ -24,6 +24,7 @@ class ModelShape:
     K: int = 4            # drafting heads (Section 3.2)
     n_sal: int = 2        # staged adaptation layers (Section 3.1)
     aeb_layers: int = 1   # self-attention layers in the Auto-embedding Block
+    lm_rank: int = 0      # 0: full drafting vocabulary heads; r > 0: each head is B[V, r] . A[r, d] (Appendix A.2.4)
     topk: Tuple[int, ...] = (10, 10, 10, 10)   # candidates kept per head
     n_nodes: int = 64     # tree nodes including the root
     prompt_len: int = 512
@@ -58,6 +59,9 @@ SHAPES = {
     # multi-pass profiler captures of single kernels at realistic sizes.
     "7b_l2": ModelShape("7b_l2", 2, 4096, 32, 128, 11008, 32000, "bf16",
                         n_nodes=64, prompt_len=2048, steps=8),
+    # 7B shape with the drafting heads factored at rank 256 (Appendix A.2.4)
+    "7b_lr256": ModelShape("7b_lr256", 32, 4096, 32, 128, 11008, 32000, "bf16", lm_rank=256,
+                           n_nodes=64, prompt_len=512, steps=128),
     "13b": ModelShape("13b", 40, 5120, 40, 128, 13824, 32000, "bf16",
                       n_nodes=64, prompt_len=1024, steps=128),
     "33b": ModelShape("33b", 60, 6656, 52, 128, 17920, 32000, "bf16",

@@ -148,7 +148,11 @@ def weight_specs(shape: ModelShape) -> List[Tuple[str, Tuple[int, ...], str]]:
         for w in ("wq", "wk", "wv", "wo"):
             specs.append((f"draft.aeb.{l}.{w}", (d, d), "normal"))
     for k in range(K):
-        specs.append((f"draft.lm_head.{k}", (v, d), "normal"))
+        if shape.lm_rank > 0:                      # two low-rank factors instead of the [V, d] matrix
+            specs.append((f"draft.lm_head.{k}.a", (shape.lm_rank, d), "normal"))
+            specs.append((f"draft.lm_head.{k}.b", (v, shape.lm_rank), "normal"))
+        else:
+            specs.append((f"draft.lm_head.{k}", (v, d), "normal"))
     return specs
 
 

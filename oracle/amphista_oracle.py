@@ -302,7 +302,11 @@ class Oracle:
         attn_o = Hp
         for l in range(s.aeb_layers):                                 # Eq. 5
             attn_o = self.aeb(attn_o, l)
-        d_logits = torch.stack([self.W(f"draft.lm_head.{k}") @ self.st(attn_o[k]) for k in range(K)])  # Eq. 6
+        if s.lm_rank > 0:      # Appendix A.2.4: the head's matrix replaced by two low-rank factors, logits = B (A x)
+            d_logits = torch.stack([self.W(f"draft.lm_head.{k}.b") @ self.st(self.W(f"draft.lm_head.{k}.a") @ self.st(attn_o[k]))
+                                    for k in range(K)])
+        else:
+            d_logits = torch.stack([self.W(f"draft.lm_head.{k}") @ self.st(attn_o[k]) for k in range(K)])  # Eq. 6
         ids, vals = [], []
         for k in range(K):
             i, v = topk_desc(d_logits[k], s.topk[k])

@@ -33,7 +33,8 @@ class amph_config(C.Structure):
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float),
                 ("weight_dtype", C.c_int32), ("kv_dtype", C.c_int32), ("max_ctx", C.c_int32),
                 ("max_batch", C.c_int32), ("K", C.c_int32), ("n_sal", C.c_int32),
-                ("aeb_layers", C.c_int32), ("topk", C.c_int32 * AMPH_MAX_HEADS_K), ("flags", C.c_int32)]
+                ("aeb_layers", C.c_int32), ("topk", C.c_int32 * AMPH_MAX_HEADS_K), ("flags", C.c_int32),
+                ("lm_rank", C.c_int32)]
 
 
 class amph_tree(C.Structure):
@@ -111,6 +112,7 @@ def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0) -> amph_co
     c.max_ctx = int(max_ctx or shape.ctx_capacity)
     c.max_batch = 1
     c.K, c.n_sal, c.aeb_layers = shape.K, shape.n_sal, shape.aeb_layers
+    c.lm_rank = getattr(shape, "lm_rank", 0)
     for k in range(shape.K):
         c.topk[k] = shape.topk[k]
     c.flags = flags

@@ -39,7 +39,7 @@ struct Layout {
   size_t state, tree, meta_v, meta_s, kv_tab, inv_freq, rope_v, rope_s;
   size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals, topk_cand;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
-  size_t xn, q, att, act, cat, last_act, ao_act, aeb_act;
+  size_t xn, q, att, act, cat, last_act, ao_act, aeb_act, lr_act;
   size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
   size_t partial_floats;
   int attn_splits;
@@ -70,7 +70,8 @@ struct amph_ctx {
   const void* mlp_w[kMaxK];
   const void* mlp_b[kMaxK];
   const void* aeb_w[2][4];
-  const void* draft_lm[kMaxK];
+  const void* draft_lm[kMaxK];      // [V, d] heads, or with lm_rank > 0 the [V, r] factors
+  const void* draft_lm_a[kMaxK];    // [r, d] factors (lm_rank > 0)
   Phase phase;
   int ctx_hi;               // host-side upper bound of the committed length
   std::string err;
@@ -147,6 +148,7 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   if (c->K < 1 || c->K > kMaxK) return fail(nullptr, AMPH_ERR_SHAPE, "K must be in 1..%d", kMaxK);
   if (c->n_sal != 1 && c->n_sal != 2) return fail(nullptr, AMPH_ERR_SHAPE, "n_sal must be 1 or 2");
   if (c->aeb_layers != 1 && c->aeb_layers != 2) return fail(nullptr, AMPH_ERR_SHAPE, "aeb_layers must be 1 or 2");
+  if (c->lm_rank < 0 || c->lm_rank > c->d_model || c->lm_rank % 8) return fail(nullptr, AMPH_ERR_SHAPE, "lm_rank must be 0 or a multiple of 8 up to d_model");
   for (int k = 0; k < c->K; ++k)
     if (c->topk[k] < 1 || c->topk[k] > kTopkStride || c->topk[k] > c->vocab)
       return fail(nullptr, AMPH_ERR_SHAPE, "topk[%d] = %d out of range 1..%d", k, c->topk[k], kTopkStride);
@@ -216,6 +218,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.last_act = l.take(esz * 16 * d);
   l.ao_act = l.take(esz * 16 * d);
   l.aeb_act = l.take(esz * 16 * d);
+  l.lr_act = l.take(esz * 16 * (size_t)(c.lm_rank > 0 ? c.lm_rank : 8));
   size_t big = 3 * d > 2 * F ? 3 * d : 2 * F;
   size_t pf = 4 * (size_t)Mcap * big;                       // room for 4 K-splits of the widest projection
   if (2 * (size_t)Mcap * V > pf) pf = 2 * (size_t)Mcap * V;
@@ -286,7 +289,12 @@ amph_status resolve(amph_ctx* ctx) {
   for (int k = 0; k < c.K; ++k) {
     ctx->mlp_w[k] = find(ctx, "draft.mlp." + std::to_string(k) + ".w", d, d, &ok);
     ctx->mlp_b[k] = find(ctx, "draft.mlp." + std::to_string(k) + ".b", d, 0, &ok);
-    ctx->draft_lm[k] = find(ctx, "draft.lm_head." + std::to_string(k), V, d, &ok);
+    if (c.lm_rank > 0) {
+      ctx->draft_lm_a[k] = find(ctx, "draft.lm_head." + std::to_string(k) + ".a", c.lm_rank, d, &ok);
+      ctx->draft_lm[k] = find(ctx, "draft.lm_head." + std::to_string(k) + ".b", V, c.lm_rank, &ok);
+    } else {
+      ctx->draft_lm[k] = find(ctx, "draft.lm_head." + std::to_string(k), V, d, &ok);
+    }
   }
   ctx->pe = find(ctx, "draft.pe", c.K, d, &ok);
   static const char* names[4] = {"wq", "wk", "wv", "wo"};
@@ -300,11 +308,11 @@ amph_status resolve(amph_ctx* ctx) {
 
 // ---- projections --------------------------------------------------------------------------
 // Y = X W^T for up to four weight matrices that share X; the result is left as fp32 partial sums.
-enum XBuf { XB_XN = 0, XB_ATT, XB_ACT, XB_CAT, XB_LAST, XB_AO, XB_AEB, XB_COUNT };
+enum XBuf { XB_XN = 0, XB_ATT, XB_ACT, XB_CAT, XB_LAST, XB_AO, XB_AEB, XB_LR, XB_COUNT };
 
 void* xbuf_ptr(amph_ctx* ctx, int xb) {
   const Layout& l = ctx->lay;
-  const size_t off[XB_COUNT] = {l.xn, l.att, l.act, l.cat, l.last_act, l.ao_act, l.aeb_act};
+  const size_t off[XB_COUNT] = {l.xn, l.att, l.act, l.cat, l.last_act, l.ao_act, l.aeb_act, l.lr_act};
   return ctx->ws + off[xb];
 }
 
@@ -509,7 +517,15 @@ amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
                       c.K, c.d_model, st);
     }
   }
-  P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                               // Eq. 6
+  if (c.lm_rank > 0) {                                                                                // Appendix A.2.4
+    P = project(ctx, XB_AO, ctx->draft_lm_a, c.K, c.lm_rank, c.d_model, c.K);
+    { ProfScope ps(ctx, AMPH_PROF_OTHER);
+    launch_gather_diag(P, ctx->ws + l.lr_act, ctx->dtype, c.K, c.lm_rank, st);
+    }
+    P = project(ctx, XB_LR, ctx->draft_lm, c.K, c.vocab, c.lm_rank, c.K);
+  } else {
+    P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                             // Eq. 6
+  }
   { ProfScope ps(ctx, AMPH_PROF_SELECT);
   launch_topk_heads(P, c.vocab, c.K, c.topk, ctx->at<int>(l.topk_ids), ctx->at<float>(l.topk_vals),
                     ctx->at<float>(l.d_logits), ctx->at<float>(l.topk_cand), st);
@@ -690,8 +706,9 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
   if (!ctx->tc && c.weight_dtype == AMPH_DTYPE_BF16 && !(c.flags & AMPH_FLAG_NO_TENSOR_CORE)) {
     void* xb[XB_COUNT];
     for (int i = 0; i < XB_COUNT; ++i) xb[i] = xbuf_ptr(ctx, i);
-    const int xrows[XB_COUNT] = {ctx->Mcap, ctx->Mcap, ctx->Mcap, ctx->Mcap, 16, 16, 16};
-    const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model};
+    const int xrows[XB_COUNT] = {ctx->Mcap, ctx->Mcap, ctx->Mcap, ctx->Mcap, 16, 16, 16, 16};
+    const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model,
+                                 c.lm_rank > 0 ? c.lm_rank : 8};
     ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
   }
   const Layout& l = ctx->lay;

@@ -159,6 +159,8 @@ void launch_mlp_heads(PartialView P, const float* last, const void* const* bias,
 // unmasked attention across the K rows, one block per attention head (Eq. 5)
 void launch_aeb_attention(PartialView P, void* out_act, int dtype, int K, int n_heads, int head_dim,
                           cudaStream_t st);
+// out_act[k][j] = P(row k, column k * r + j): row k of the k-th low-rank projection, as the next projection's input
+void launch_gather_diag(PartialView P, void* out_act, int dtype, int K, int r, cudaStream_t st);
 // per head k: top-c_k of row k of segment k; also stores the row into d_logits[k]
 // cand: scratch for the slices' candidates, kMaxK * kTopkCandChunks * kTopkStride (value, id) pairs
 constexpr int kTopkCandChunks = 32;

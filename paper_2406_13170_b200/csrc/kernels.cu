@@ -647,6 +647,18 @@ void launch_gather_last(const float* h1, const float* h2, const DevState* st_dev
   AMPH_DISPATCH(dtype, launch_pdl(gather_last_kernel<T>, dim3(2, gy), dim3(256), 0, st, h1, h2, st_dev, last, (T*)last_act, d));
 }
 
+template <typename T>
+__global__ void gather_diag_kernel(PartialView P, T* __restrict__ out, int r) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int k = blockIdx.x;
+  for (int j = threadIdx.x; j < r; j += blockDim.x) out[(size_t)k * r + j] = from_f<T>(sum_partials(P, k, k * r + j));
+}
+
+void launch_gather_diag(PartialView P, void* out_act, int dtype, int K, int r, cudaStream_t st) {
+  AMPH_DISPATCH(dtype, launch_pdl(gather_diag_kernel<T>, dim3(K), dim3(256), 0, st, P, (T*)out_act, r));
+}
+
 struct BiasPtrs { const void* b[kMaxK]; };
 
 template <typename T>

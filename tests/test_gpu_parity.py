@@ -19,7 +19,7 @@ def _setup(shape, topo, flags=0, max_ctx=None):
     from paper_2406_13170_b200 import Amphista
     w_cpu = inputs.make_weights(shape, seed=0)
     w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
-    for k in ("tok_emb", "layers.0.wq", "draft.lm_head.1"):
+    for k in ("tok_emb", "layers.0.wq", "draft.lm_head.1.b" if shape.lm_rank else "draft.lm_head.1"):
         assert torch.equal(w_cpu[k], w_gpu[k].cpu()), "input generator must be device independent"
     model = Amphista(shape, topo, w_gpu, max_ctx=max_ctx, flags=flags)
     orc = ao.Oracle(shape, w_cpu, dtype=torch.float64)
@@ -87,13 +87,16 @@ def test_long_prompt_many_attention_splits_bf16():
     model.close()
 
 
-@pytest.mark.parametrize("variant", [dict(n_sal=1), dict(aeb_layers=2), dict(n_sal=1, aeb_layers=2)],
-                         ids=["one-sal", "alpha-two-aeb-layers", "one-sal-two-aeb-layers"])
+@pytest.mark.parametrize("variant", [dict(n_sal=1), dict(aeb_layers=2), dict(n_sal=1, aeb_layers=2), dict(lm_rank=64),
+                                     dict(lm_rank=24)],
+                         ids=["one-sal", "alpha-two-aeb-layers", "one-sal-two-aeb-layers", "low-rank-heads-64",
+                              "low-rank-heads-24"])
 @pytest.mark.parametrize("base", ["tiny", "small_bf16"])
 def test_draft_module_variants(base, variant):
     """The draft-module variants the paper evaluates: a single adaptation layer (the "One-Adaptation-Layer"
-    ablation of Section 4.5: every head then reads h1) and the two-layer Auto-embedding Block ("Amphista-alpha",
-    Appendix A.2.3)."""
+    ablation of Section 4.5: every head then reads h1), the two-layer Auto-embedding Block ("Amphista-alpha",
+    Appendix A.2.3) and vocabulary heads factored into two low-rank matrices (Appendix A.2.4; on bf16, rank 64
+    takes the tensor-core projection and rank 24 the plain one)."""
     shape = inputs.get_shape(base).with_(**variant)
     topo = inputs.make_tree(shape.n_nodes, shape.topk)
     model, orc = _setup(shape, topo)

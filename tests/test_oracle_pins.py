@@ -479,3 +479,25 @@ def test_variants_stay_lossless(variant):
         emitted = orc.step(st, t, _plant(t, st.root, ref[len(out) + 1: len(out) + 1 + t.depth[leaf]], leaf), {})
         out += emitted
     assert out == ref[: len(out)] and st.root == ref[len(out)]
+
+
+def test_variant_low_rank_lm_heads_equal_the_product_matrix():
+    """Appendix A.2.4 replaces each head's [V, d] matrix by two low-rank factors: the draft logits must be
+    those of a full head whose matrix is the product B.A, and the factors hold (V + d) r parameters each."""
+    r = 8
+    shape = MICRO.with_(lm_rank=r)
+    w = inputs.make_weights(shape, seed=0, std=0.2)
+    specs = {n: shp for n, shp, _ in inputs.weight_specs(shape)}
+    assert specs["draft.lm_head.0.a"] == (r, MICRO.d_model) and specs["draft.lm_head.0.b"] == (MICRO.vocab, r)
+    assert "draft.lm_head.0" not in specs
+    full = {k: v for k, v in w.items() if ".lm_head." not in k or k == "lm_head"}
+    for k in range(MICRO.K):
+        full[f"draft.lm_head.{k}"] = (w[f"draft.lm_head.{k}.b"].double() @ w[f"draft.lm_head.{k}.a"].double())
+    lo = ao.Oracle(shape, w, dtype=torch.float64)
+    hi = ao.Oracle(MICRO, full, dtype=torch.float64)
+    prompt = inputs.make_prompt(MICRO).tolist()
+    ids_l, vals_l, dl_l = lo.draft(lo.prefill(prompt))
+    ids_h, vals_h, dl_h = hi.draft(hi.prefill(prompt))
+    assert torch.allclose(dl_l, dl_h, atol=1e-10)
+    assert [list(map(int, i)) for i in ids_l] == [list(map(int, i)) for i in ids_h]
+    assert torch.linalg.matrix_rank(full["draft.lm_head.0"]).item() == r
