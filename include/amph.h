@@ -52,7 +52,8 @@ enum { AMPH_DTYPE_F32 = 0, AMPH_DTYPE_BF16 = 1 };
 /* amph_config.flags */
 enum {
   AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
-  AMPH_FLAG_NO_GRAPH = 2        /* launch kernels one by one instead of replaying a CUDA graph */
+  AMPH_FLAG_NO_GRAPH = 2,       /* launch kernels one by one instead of replaying a CUDA graph */
+  AMPH_FLAG_NO_SIDE_PREFETCH = 4 /* no second stream: do not prefetch weights into L2 while attention runs */
 };
 
 #define AMPH_MAX_HEADS_K 8
