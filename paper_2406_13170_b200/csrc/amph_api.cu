@@ -412,7 +412,8 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
   launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
-                        c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr);
+                        c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr,
+                        (c.flags & AMPH_FLAG_SEPARATE_MERGE) != 0);
   }
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);

@@ -133,10 +133,12 @@ struct AttnScratch {
 };
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out,
                            int dtype, int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi,
-                           int max_splits, cudaStream_t st, int early = 0);
+                           int max_splits, cudaStream_t st, int early = 0, int separate_merge = 0);
 
-void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
-                               int head_dim, int max_ctx, int splits, cudaStream_t st);
+// merged_out != NULL and splits <= 8: the splits of a head run as one cluster and write the final bf16 rows to
+// merged_out themselves (returns true); otherwise partial results go to sc for attn_combine_kernel (returns false).
+bool launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
+                               int head_dim, int max_ctx, int splits, cudaStream_t st, void* merged_out);
 
 void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale(),
                    int early = 0);

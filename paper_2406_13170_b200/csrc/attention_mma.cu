@@ -6,6 +6,11 @@
 // (16-byte chunks, XOR-swizzled so that ldmatrix is bank-conflict free).  Scores, the online softmax and
 // the output accumulator stay in registers; each CTA leaves an unnormalised partial output plus the
 // running (max, sum) per row, merged by attn_combine_kernel.
+//
+// Merge in the same launch (MERGE = true): the KV splits of one head form a thread-block cluster (up to 8).
+// Each CTA parks its partial output in its own shared memory; after a cluster barrier CTA j merges rows
+// j, j + S, ... of all S partials through distributed shared memory and writes the final bf16 rows, so the
+// partials never travel through L2 and the merge kernel with its launch boundary disappears.
 #include <math.h>
 
 #include "amph_internal.cuh"
@@ -63,11 +68,31 @@ __device__ __forceinline__ void load_tile(bf16* dst, const bf16* src, int s0, in
   }
 }
 
-template <int DH>
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in the CTA of rank `rank` of this cluster
+__device__ __forceinline__ uint32_t peer_smem(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_peer4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_peer2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
+template <int DH, bool MERGE>
 __global__ void __launch_bounds__(kThreads)
 tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, const bf16* __restrict__ vc,
                      const RowMeta* __restrict__ meta, float* __restrict__ po, float* __restrict__ pml,
-                     int rows_cap, int n_heads, int max_ctx) {
+                     int rows_cap, int n_heads, int max_ctx, bf16* __restrict__ out) {
   pdl_wait();
   pdl_launch_dependents();
   constexpr int KS = DH / 16;                        // k-steps over the head dimension
@@ -224,6 +249,53 @@ tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, co
   }
   if (n_tiles == 0) cp_async_wait<0>();
 
+  if constexpr (MERGE) {
+    // ---- park the partial output and (max, sum) in shared memory (the K / V ring is free now)
+    float* Os = reinterpret_cast<float*>(Ks);                        // [64][DH]
+    float* MLs = Os + kRows * DH;                                    // [64][2]
+    const int la = warp * 16 + g, lb = la + 8;
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      *reinterpret_cast<float2*>(Os + la * DH + i * 8 + 2 * t) = make_float2(oacc[i][0], oacc[i][1]);
+      *reinterpret_cast<float2*>(Os + lb * DH + i * 8 + 2 * t) = make_float2(oacc[i][2], oacc[i][3]);
+    }
+    if (t == 0) {
+      *reinterpret_cast<float2*>(MLs + la * 2) = make_float2(m_a, l_a);
+      *reinterpret_cast<float2*>(MLs + lb * 2) = make_float2(m_b, l_b);
+    }
+    cluster_sync_all();
+    // ---- CTA `split` of the S in the cluster merges rows split, split + S, ...; one warp per row, a lane per 4 columns
+    const int S = gridDim.y;
+    const uint32_t os0 = smem_u32(Os), ml0 = smem_u32(MLs);
+    for (int r = split + S * warp; r < kRows; r += S * (kThreads / 32)) {
+      const int gr = rb * kRows + r;
+      if (gr >= rows_cap) continue;
+      float2 ml = make_float2(-INFINITY, 0.f);
+      if (lane < S) ml = ld_peer2(peer_smem(ml0 + (uint32_t)r * 8, (uint32_t)lane));
+      float M = ml.x;
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      const float wgt = ml.x == -INFINITY ? 0.f : expf(ml.x - M);     // lane s holds the weight of split s
+      float den = ml.y * wgt;
+      for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < S; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, wgt, s);
+        if (lane * 4 < DH && ws != 0.f) {
+          const float4 v = ld_peer4(peer_smem(os0 + (uint32_t)(r * DH + lane * 4) * 4, (uint32_t)s));
+          acc.x += v.x * ws; acc.y += v.y * ws; acc.z += v.z * ws; acc.w += v.w * ws;
+        }
+      }
+      if (lane * 4 < DH) {
+        const float inv = den > 0.f ? 1.0f / den : 0.f;
+        uint2 u;
+        u.x = pack_bf16(acc.x * inv, acc.y * inv);
+        u.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(out + (size_t)gr * n_heads * DH + h * DH + lane * 4) = u;
+      }
+    }
+    cluster_sync_all();                              // nobody leaves while a peer may still read its shared memory
+    return;
+  }
   // ---- partial results
   const size_t oa = ((size_t)split * n_heads + h) * rows_cap + row_a;
   const size_t ob = oa + 8;
@@ -242,21 +314,45 @@ tree_attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, co
 }
 
 template <int DH>
-void launch_t(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads, int max_ctx,
-              int splits, cudaStream_t st) {
+bool launch_t(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads, int max_ctx,
+              int splits, cudaStream_t st, void* merged_out) {
   const size_t smem = sizeof(bf16) * (kRows * DH + 4 * kKeys * DH);
-  cudaFuncSetAttribute(tree_attn_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid(n_heads, splits, (rows + kRows - 1) / kRows);
-  launch_pdl(tree_attn_mma_kernel<DH>, dim3(grid), dim3(kThreads), smem, st, (const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v, meta, sc.o,
-                                                        sc.ml, rows, n_heads, max_ctx);
+  if (merged_out != nullptr && splits <= 8) {
+    // the KV splits of a head as one cluster; merge through distributed shared memory
+    static_assert(sizeof(float) * (kRows * DH + kRows * 2) <= sizeof(bf16) * 4 * kKeys * DH, "partial output must fit the K / V ring");
+    cudaFuncSetAttribute(tree_attn_mma_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = 1;
+    at[1].val.clusterDim.y = splits;
+    at[1].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 2;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attn_mma_kernel<DH, true>, (const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v,
+                                             meta, sc.o, sc.ml, rows, n_heads, max_ctx, (bf16*)merged_out);
+    if (e == cudaSuccess) return true;
+    cudaGetLastError();                              // cluster launch refused: fall back to two launches
+  }
+  cudaFuncSetAttribute(tree_attn_mma_kernel<DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  launch_pdl(tree_attn_mma_kernel<DH, false>, dim3(grid), dim3(kThreads), smem, st, (const bf16*)q, (const bf16*)kv.k, (const bf16*)kv.v, meta, sc.o,
+                                                        sc.ml, rows, n_heads, max_ctx, (bf16*)nullptr);
+  return false;
 }
 
 }  // namespace
 
-void launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
-                               int head_dim, int max_ctx, int splits, cudaStream_t st) {
-  if (head_dim == 64) launch_t<64>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st);
-  else launch_t<128>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st);
+bool launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
+                               int head_dim, int max_ctx, int splits, cudaStream_t st, void* merged_out) {
+  if (head_dim == 64) return launch_t<64>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st, merged_out);
+  return launch_t<128>(q, kv, meta, sc, rows, n_heads, max_ctx, splits, st, merged_out);
 }
 
 }  // namespace amph

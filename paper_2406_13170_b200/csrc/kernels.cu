@@ -481,12 +481,14 @@ static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, Attn
 
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out, int dtype,
                            int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi, int max_splits,
-                           cudaStream_t st, int early) {
+                           cudaStream_t st, int early, int separate_merge) {
   int splits = (ctx_hi + 127) / 128;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
   if (dtype == AMPH_DTYPE_BF16) {                    // tensor-core path; the kernel below serves fp32 caches
-    launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st);
+    if (launch_tree_attention_mma(q, kv, meta, sc, rows, n_heads, head_dim, max_ctx, splits, st,
+                                  separate_merge ? nullptr : out))
+      return;
     launch_pdl(attn_combine_kernel<bf16>, dim3(dim3(rows, n_heads)), dim3(head_dim < 128 ? 64 : 128), 0, st, sc.o, sc.ml, (bf16*)out, splits,
                                                                                         rows, n_heads, head_dim, early);
     return;
