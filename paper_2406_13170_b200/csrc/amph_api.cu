@@ -229,7 +229,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.partial_floats = pf;
   l.partial = l.take(4 * pf);
   int splits = (296 + c.n_heads - 1) / c.n_heads;
-  if (splits > 16) splits = 16;
+  if (splits > 8) splits = 8;                               // the KV splits of a head run as one thread-block cluster (<= 8 CTAs)
   l.attn_splits = splits;
   l.att_o = l.take(4 * (size_t)splits * c.n_heads * Mcap * c.head_dim);
   l.att_ml = l.take(4 * (size_t)splits * c.n_heads * Mcap * 2);
@@ -746,7 +746,7 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
     const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model,
                                  c.lm_rank > 0 ? c.lm_rank : 8};
     ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
-    if (ctx->tc && !ctx->side && ctx->stream != nullptr && !(c.flags & AMPH_FLAG_NO_SIDE_PREFETCH)) {
+    if (ctx->tc && !ctx->side && ctx->stream != nullptr && (c.flags & AMPH_FLAG_SIDE_PREFETCH)) {
       if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
           cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
           cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {

@@ -26,7 +26,7 @@ namespace {
 constexpr int kTileM = 128;           // weight rows per CTA (UMMA M)
 constexpr int kTileK = 64;            // bf16 elements per 128-byte swizzle row
 constexpr int kUmmaK = 16;            // K per tcgen05.mma for 16-bit inputs
-constexpr int kStageKb = 2;           // 64-wide K blocks fetched by one TMA copy (one pipeline stage)
+constexpr int kStageKb = 2;           // 64-wide K blocks fetched by one TMA copy (one pipeline stage) when both operands' stage fits twice per CTA
 constexpr int kMaxSeg = 8;
 constexpr int kThreads = 192;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // a barrier wait gives up after one second
@@ -47,6 +47,7 @@ struct TcParams {
   int rows;                 // live rows (only these are stored)
   int stages;
   int l2_prefetch;          // weight tiles (beyond the ring) each CTA pulls into L2 before it waits
+  int ks;                   // K blocks per stage (depth of the tensor maps' boxes): kStageKb, or 1 for many activation rows
   int* err_flag;
 };
 
@@ -159,16 +160,17 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
   const int row0 = (tile - seg * prm.tiles_per_seg) * kTileM;       // first weight row of this tile
-  // K range of this split in whole stages (kStageKb blocks), so that every copy starts on a stage boundary
-  const int units = (prm.kblocks + kStageKb - 1) / kStageKb;
-  const int kb_lo = (int)((long long)split * units / prm.splits) * kStageKb;
-  int kb_hi = (int)((long long)(split + 1) * units / prm.splits) * kStageKb;
+  // K range of this split in whole stages (ks blocks), so that every copy starts on a stage boundary
+  const int ks = prm.ks;
+  const int units = (prm.kblocks + ks - 1) / ks;
+  const int kb_lo = (int)((long long)split * units / prm.splits) * ks;
+  int kb_hi = (int)((long long)(split + 1) * units / prm.splits) * ks;
   if (kb_hi > prm.kblocks) kb_hi = prm.kblocks;
   const int nkb = kb_hi - kb_lo;
-  const int nit = (nkb + kStageKb - 1) / kStageKb;                  // pipeline iterations
+  const int nit = (nkb + ks - 1) / ks;                  // pipeline iterations
   const int nt = prm.nt, stages = prm.stages;
   const uint32_t a_tile = kTileM * kTileK * 2, b_tile = (uint32_t)nt * kTileK * 2;     // one K block of each operand
-  const uint32_t a_bytes = kStageKb * a_tile, b_bytes = kStageKb * b_tile;
+  const uint32_t a_bytes = ks * a_tile, b_bytes = ks * b_tile;
   const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint32_t tmem_cols = 32;
@@ -204,16 +206,16 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     if (leader) {
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
-        tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * kStageKb, &full_bar[i]);
+        tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
-      for (int i = npre; i < npf; ++i) tma_prefetch_l2_3d(wmap, row0, kb_lo + i * kStageKb);
+      for (int i = npre; i < npf; ++i) tma_prefetch_l2_3d(wmap, row0, kb_lo + i * ks);
     }
     __syncwarp();
     pdl_wait();
     if (leader)
       for (int i = 0; i < npre; ++i)
-        tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[i]);
+        tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[i]);
     __syncwarp();
     int issued = npre;
     for (int i = npre; i < nit; ++i) {
@@ -222,8 +224,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        tma_load_3d(a, wmap, row0, kb_lo + i * kStageKb, &full_bar[s]);
-        tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * kStageKb, &full_bar[s]);
+        tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
+        tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[s]);
       }
       __syncwarp();
       issued = i + 1;
@@ -248,7 +250,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       if (leader) {
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-        const int nk = nkb - i * kStageKb < kStageKb ? nkb - i * kStageKb : kStageKb;   // blocks of the stage inside the K range
+        const int nk = nkb - i * ks < ks ? nkb - i * ks : ks;   // blocks of the stage inside the K range
         for (int kk = 0; kk < nk; ++kk) {
           const uint64_t adesc = umma_desc(a_addr + (uint32_t)kk * a_tile), bdesc = umma_desc(a_addr + a_bytes + (uint32_t)kk * b_tile);
 #pragma unroll
@@ -311,19 +313,19 @@ struct TcGemm {
   int n_x = 0;
   void* xptr[16];
   int xrows[16], xcols[16];
-  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;   // (ptr, rows, cols, box rows)
+  std::map<std::tuple<const void*, int, int, int, int>, CUtensorMap> cache;   // (ptr, rows, cols, box rows, box K blocks)
   int sm_count = 148;
   int max_smem = 0;
 
-  const CUtensorMap* get(const void* ptr, int rows, int cols, int box_rows) {
-    auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  const CUtensorMap* get(const void* ptr, int rows, int cols, int box_rows, int box_kb = kStageKb) {
+    auto key = std::make_tuple(ptr, rows, cols, box_rows, box_kb);
     auto it = cache.find(key);
     if (it != cache.end()) return &it->second;
     CUtensorMap m;
     // (column within a K block, row, K block): stride of a row = its pitch, of a K block = 128 bytes
     const cuuint64_t dims[3] = {(cuuint64_t)kTileK, (cuuint64_t)rows, (cuuint64_t)cols / kTileK};
     const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)kTileK * 2};
-    const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows, (cuuint32_t)kStageKb};
+    const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows, (cuuint32_t)box_kb};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -369,7 +371,9 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   // K-splits: fill about two CTAs per SM, keep at least four 64-wide K blocks per CTA
   int splits = (2 * g->sm_count) / tiles;
   if (splits > kblocks / 4) splits = kblocks / 4;
-  if (splits > (kblocks + kStageKb - 1) / kStageKb) splits = (kblocks + kStageKb - 1) / kStageKb;
+  // many activation rows: a two-block stage would leave room for one CTA per SM only, so stage single blocks
+  const int ks = nt <= 64 ? kStageKb : 1;
+  if (splits > (kblocks + ks - 1) / ks) splits = (kblocks + ks - 1) / ks;
   if (splits > 16) splits = 16;
   while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
   if (splits < 1) splits = 1;
@@ -378,14 +382,14 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   memset(&pack, 0, sizeof pack);
   for (int s = 0; s < n_seg; ++s) {
     if ((uintptr_t)w[s] & 15) return false;
-    const CUtensorMap* m = g->get(w[s], out, in, kTileM);
+    const CUtensorMap* m = g->get(w[s], out, in, kTileM, ks);
     if (!m) return false;
     pack.w[s] = *m;
   }
-  const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt);
+  const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt, ks);
   if (!mx) return false;
   pack.x = *mx;
-  const uint32_t stage_bytes = kStageKb * kTileM * kTileK * 2 + ((kStageKb * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  const uint32_t stage_bytes = ks * kTileM * kTileK * 2 + ((ks * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
   int stages = (int)((110 * 1024) / stage_bytes);          // <= ~110 KB per CTA: two CTAs per SM
   if (stages > 8) stages = 8;
   if (stages < 2) stages = 2;
@@ -399,10 +403,11 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.nt = nt;
   prm.rows = rows;
   prm.stages = stages;
+  prm.ks = ks;
   // about 40 MB of L2 for prefetched weight tiles, shared by the CTAs that can be resident at once
   {
     const long long resident = (long long)tiles * splits < 2LL * g->sm_count ? (long long)tiles * splits : 2LL * g->sm_count;
-    long long pf = (40LL << 20) / (resident * (kStageKb * kTileM * kTileK * 2));
+    long long pf = (40LL << 20) / (resident * (ks * kTileM * kTileK * 2));
     prm.l2_prefetch = (int)(pf > 32 ? 32 : pf);
   }
   prm.err_flag = g->err_flag;
