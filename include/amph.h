@@ -78,8 +78,10 @@ typedef struct {
   int32_t max_ctx;        /* KV capacity in slots (committed tokens + tree nodes)           */
   int32_t max_batch;      /* must be 1                                                      */
   int32_t K;              /* drafting heads, 1..AMPH_MAX_HEADS_K (the paper uses 4)         */
-  int32_t n_sal;          /* staged adaptation layers: 2 (the paper's design) or 1          */
-  int32_t aeb_layers;     /* 1 (the paper's design) or 2 (its "alpha" variant)              */
+  int32_t n_sal;          /* staged adaptation layers: 2 (the paper's design), 1, or 0 (the  *
+                           * heads then read the target's hidden state; Section 4.5)         */
+  int32_t aeb_layers;     /* 1 (the paper's design), 2 (its "alpha" variant) or 0 (no        *
+                           * Auto-embedding Block: independent heads; Section 4.5)           */
   int32_t topk[AMPH_MAX_HEADS_K]; /* candidates kept per head, each 1..AMPH_TOPK_STRIDE     */
   int32_t flags;          /* AMPH_FLAG_*                                                    */
   int32_t lm_rank;        /* 0: each drafting head owns a [vocab, d] matrix (Eq. 6); r > 0: it owns two

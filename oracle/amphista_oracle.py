@@ -293,10 +293,12 @@ class Oracle:
                                           st.sal_kv[stage - 1]))
             feats = outs
             stage_out.append(outs[-1])
+        if s.n_sal == 0:                                              # Section 4.5, "w/o Staged-Adaptation":
+            stage_out = [feats[-1]]                                   # the heads read the target's h_t itself
         st.pending = []
         rows = []
         for k in range(1, K + 1):                                     # Eq. 2: head -> stage split
-            src = stage_out[0] if (k <= K // 2 or s.n_sal == 1) else stage_out[1]
+            src = stage_out[0] if (k <= K // 2 or s.n_sal <= 1) else stage_out[1]
             rows.append(src + silu(self.W(f"draft.mlp.{k-1}.w") @ self.st(src) + self.W(f"draft.mlp.{k-1}.b")))
         Hp = torch.stack(rows) + self.W("draft.pe")                   # Eq. 3, Eq. 4
         attn_o = Hp

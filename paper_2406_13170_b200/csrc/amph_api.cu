@@ -149,8 +149,8 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   if (c->kv_dtype != c->weight_dtype) return fail(nullptr, AMPH_ERR_SHAPE, "kv_dtype must equal weight_dtype");
   if (c->max_batch != 1) return fail(nullptr, AMPH_ERR_SHAPE, "max_batch must be 1");
   if (c->K < 1 || c->K > kMaxK) return fail(nullptr, AMPH_ERR_SHAPE, "K must be in 1..%d", kMaxK);
-  if (c->n_sal != 1 && c->n_sal != 2) return fail(nullptr, AMPH_ERR_SHAPE, "n_sal must be 1 or 2");
-  if (c->aeb_layers != 1 && c->aeb_layers != 2) return fail(nullptr, AMPH_ERR_SHAPE, "aeb_layers must be 1 or 2");
+  if (c->n_sal < 0 || c->n_sal > 2) return fail(nullptr, AMPH_ERR_SHAPE, "n_sal must be 0, 1 or 2");
+  if (c->aeb_layers < 0 || c->aeb_layers > 2) return fail(nullptr, AMPH_ERR_SHAPE, "aeb_layers must be 0, 1 or 2");
   if (c->lm_rank < 0 || c->lm_rank > c->d_model || c->lm_rank % 8) return fail(nullptr, AMPH_ERR_SHAPE, "lm_rank must be 0 or a multiple of 8 up to d_model");
   for (int k = 0; k < c->K; ++k)
     if (c->topk[k] < 1 || c->topk[k] > kTopkStride || c->topk[k] > c->vocab)
@@ -533,8 +533,10 @@ amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
   }
   run_sals(ctx, ctx->at<float>(l.pend_h), ds->pend_tok, rows, ctx->ctx_hi);
   { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_gather_last(ctx->at<float>(l.h1), ctx->at<float>(c.n_sal == 2 ? l.h2 : l.h1), ds, ctx->at<float>(l.last),
-                     ctx->ws + l.last_act, ctx->dtype, c.d_model, st);
+  // without adaptation layers (the "w/o Staged-Adaptation" ablation) every head reads the target's hidden state itself
+  const float* s1 = ctx->at<float>(c.n_sal == 0 ? l.pend_h : l.h1);
+  const float* s2 = ctx->at<float>(c.n_sal == 0 ? l.pend_h : (c.n_sal == 2 ? l.h2 : l.h1));
+  launch_gather_last(s1, s2, ds, ctx->at<float>(l.last), ctx->ws + l.last_act, ctx->dtype, c.d_model, st);
   }
   PartialView P = project(ctx, XB_LAST, ctx->mlp_w, c.K, c.d_model, c.d_model, 2);                   // Eq. 2
   { ProfScope ps(ctx, AMPH_PROF_OTHER);
@@ -768,7 +770,7 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
     target_forward(ctx, M, start + nr);
     if (last) target_head(ctx, M);
     const int nrs = last ? nr - 1 : nr;           // the last prompt row stays pending for the first draft
-    if (nrs > 0) {
+    if (nrs > 0 && c.n_sal > 0) {
       rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.next_tok), prompt_ids + start + 1, sizeof(int) * nrs, cudaMemcpyHostToDevice, st), "prompt upload");
       if (rc != AMPH_OK) return rc;
       launch_meta_chain(ctx->at<RowMeta>(l.meta_s), start, nrs, st);

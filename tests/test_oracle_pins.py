@@ -501,3 +501,58 @@ def test_variant_low_rank_lm_heads_equal_the_product_matrix():
     assert torch.allclose(dl_l, dl_h, atol=1e-10)
     assert [list(map(int, i)) for i in ids_l] == [list(map(int, i)) for i in ids_h]
     assert torch.linalg.matrix_rank(full["draft.lm_head.0"]).item() == r
+
+
+def test_variant_without_adaptation_layers_or_auto_embedding():
+    """Section 4.5's ablations that remove a module.  Without adaptation layers every head's MLP reads the target's
+    last hidden state (the row the target's own head consumed) and the sampled token plays no part; without the
+    Auto-embedding Block the head rows go to their vocabulary projections unchanged."""
+    prompt = inputs.make_prompt(MICRO).tolist()
+    # -- no adaptation layers
+    s0 = MICRO.with_(n_sal=0)
+    o0 = ao.Oracle(s0, inputs.make_weights(s0, seed=0, std=0.2), dtype=torch.float64)
+    assert not any(n.startswith("draft.sal") or n.startswith("draft.fc") for n, _, _ in inputs.weight_specs(s0))
+    st = o0.prefill(prompt)
+    h_t = st.pending[-1][0].clone()
+    assert torch.allclose(o0.W("lm_head") @ h_t, st.last_logits, atol=1e-10)      # it is the row the target head consumed
+    taps = {}
+    o0.draft(st, taps)
+    base = taps["Hp"] - o0.W("draft.pe")
+    for k in range(MICRO.K):
+        w, b = o0.W(f"draft.mlp.{k}.w"), o0.W(f"draft.mlp.{k}.b")
+        assert torch.allclose(base[k], h_t + torch.nn.functional.silu(w @ h_t + b), atol=1e-12)
+    st2 = o0.prefill(prompt)                       # the sampled token is unused: change it, nothing moves
+    st2.pending = [(h, (nxt + 1) % MICRO.vocab, p) for (h, nxt, p) in st2.pending]
+    t2 = {}
+    o0.draft(st2, t2)
+    assert torch.equal(t2["Hp"], taps["Hp"])
+    # -- no Auto-embedding Block
+    s1 = MICRO.with_(aeb_layers=0)
+    o1 = ao.Oracle(s1, inputs.make_weights(s1, seed=0, std=0.2), dtype=torch.float64)
+    assert not any(n.startswith("draft.aeb") for n, _, _ in inputs.weight_specs(s1))
+    t1 = {}
+    _, _, dl = o1.draft(o1.prefill(prompt), t1)
+    assert torch.equal(t1["attn_o"], t1["Hp"])
+    for k in range(MICRO.K):
+        assert torch.allclose(dl[k], o1.W(f"draft.lm_head.{k}") @ t1["Hp"][k], atol=1e-12)
+    # a head's logits then depend on its own row only (no exchange between the heads)
+    two = ao.Oracle(MICRO, inputs.make_weights(MICRO, seed=0, std=0.2), dtype=torch.float64)
+    Hp = inputs.normal_tensor((MICRO.K, MICRO.d_model), 1.0, 9, "Hp", dtype=torch.float64)
+    Hq = Hp.clone(); Hq[0] += 1.0
+    assert bool(((two.aeb(Hq) - two.aeb(Hp)).abs().amax(dim=1)[1:] > 1e-8).all())   # with the block, rows do interact
+
+
+@pytest.mark.parametrize("variant", [dict(n_sal=0), dict(aeb_layers=0)], ids=["no-sal", "no-aeb"])
+def test_ablations_stay_lossless(variant):
+    shape = MICRO.with_(**variant)
+    orc = ao.Oracle(shape, inputs.make_weights(shape, seed=0, std=0.2), dtype=torch.float64)
+    prompt = inputs.make_prompt(shape).tolist()
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    t = _tables(topo)
+    ref = orc.greedy_ar(prompt, 4 * (shape.K + 1) + 1)
+    st = orc.prefill(prompt)
+    out = []
+    for i in range(4):
+        leaf = t.leaves[i % len(t.leaves)]
+        out += orc.step(st, t, _plant(t, st.root, ref[len(out) + 1: len(out) + 1 + t.depth[leaf]], leaf), {})
+    assert out == ref[: len(out)] and st.root == ref[len(out)]
