@@ -19,7 +19,7 @@ def _setup(shape, topo, flags=0, max_ctx=None):
     from paper_2406_13170_b200 import Amphista
     w_cpu = inputs.make_weights(shape, seed=0)
     w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
-    for k in ("tok_emb", "layers.0.wq", "draft.lm_head.1.b" if shape.lm_rank else "draft.lm_head.1"):
+    for k in ("tok_emb", "layers.0.wq", "draft.lm_head.0.b" if shape.lm_rank else "draft.lm_head.0"):
         assert torch.equal(w_cpu[k], w_gpu[k].cpu()), "input generator must be device independent"
     model = Amphista(shape, topo, w_gpu, max_ctx=max_ctx, flags=flags)
     orc = ao.Oracle(shape, w_cpu, dtype=torch.float64)
@@ -106,4 +106,45 @@ def test_draft_module_variants(base, variant):
     rep = run_parity(model, orc, shape, topo, prompt, 4, TOL_BF16 if bf else TOL_F32, TIE_BF16 if bf else TIE_F32, True)
     print(rep)
     assert rep.steps == 4 and max(rep.accepted) >= 3
+    model.close()
+
+
+@pytest.mark.parametrize("case", ["root-only-tree", "one-token-prompt", "max-nodes-128", "one-head", "eight-heads-top16"])
+def test_degenerate_and_maximum_shapes(case):
+    """The corners of the interface: a tree that is only its root (every step then emits exactly one token, i.e.
+    plain autoregressive decoding through the speculative path), a prompt of one token, the largest tree the
+    library takes (128 nodes: two 64-row blocks in attention, 128 activation rows in the projections), a single
+    drafting head, and the maximum of eight heads keeping 16 candidates each."""
+    base = inputs.get_shape("tiny")
+    if case == "root-only-tree":
+        shape, topo, steps, planted = base.with_(n_nodes=1), inputs.chain_tree(1), 6, False
+    elif case == "one-token-prompt":
+        shape, steps, planted = base.with_(prompt_len=1), 5, True
+        topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    elif case == "max-nodes-128":
+        shape = base.with_(n_nodes=128, topk=(16, 8, 4, 2))
+        topo, steps, planted = inputs.make_tree(128, shape.topk), 4, True
+    elif case == "one-head":
+        shape = base.with_(K=1, topk=(4,), n_nodes=5)
+        topo, steps, planted = inputs.make_tree(5, shape.topk), 5, True
+    else:
+        shape = base.with_(K=8, topk=(16,) * 8, n_nodes=96)
+        topo, steps, planted = inputs.make_tree(96, shape.topk), 3, True
+    model, orc = _setup(shape, topo)
+    prompt = inputs.make_prompt(shape).tolist()
+    rep = run_parity(model, orc, shape, topo, prompt, steps, TOL_F32, TIE_F32, planted)
+    print(rep)
+    assert rep.steps == steps
+    if case == "root-only-tree":
+        assert rep.accepted == [1] * steps
+    model.close()
+
+
+def test_small_bf16_max_nodes_128():
+    """128 tree rows on the tensor-core path: single-block stages in the projections, two row blocks per attention cluster."""
+    shape = inputs.get_shape("small_bf16").with_(n_nodes=128, topk=(16, 8, 4, 2))
+    topo = inputs.make_tree(128, shape.topk)
+    model, orc = _setup(shape, topo)
+    rep = run_parity(model, orc, shape, topo, inputs.make_prompt(shape).tolist(), 3, TOL_BF16, TIE_BF16, True)
+    print(rep)
     model.close()
