@@ -172,7 +172,8 @@ amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int3
 amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n);
 
 /* Debug taps (stream-ordered copy into dst, host or device).  Names and element types:
- *   "hidden" f32 [n_nodes,d] post-final-norm rows of the last verify; "logits" f32 [n_nodes,V];
+ *   "hidden" f32 [rows,d] post-final-norm rows of the last target pass and "logits" f32 [rows,V] (rows =
+ *   n_nodes after amph_verify_tree; after amph_prefill the rows of its last chunk of AMPH_MAX_NODES prompt tokens);
  *   "d_logits" f32 [K,V]; "hp" f32 [K,d] (Eq. 4); "attn_o" f32 [K,d] (Eq. 5);
  *   "sal_h" f32 [2,d] (Eq. 1: h^1_t, h^2_t of the last row); "tree_tokens", "argmax" i32 [n_nodes];
  *   "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v": f32 [rows, d] for cache slots 0..rows-1,

@@ -55,7 +55,8 @@ struct amph_ctx {
   cudaStream_t stream;
   int dtype;
   size_t esz;
-  int Mcap;                 // rows carried by a verification / prefill-chunk pass
+  int Mcap;                 // row capacity of the activation buffers = rows of a prefill chunk
+  int Mver;                 // rows carried by a verification pass (tree nodes rounded up to 16)
   int rows_small;           // rows carried by the draft module's passes
   Layout lay;
   char* ws;
@@ -185,8 +186,13 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   return AMPH_OK;
 }
 
-void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, size_t* kv_bytes) {
-  const int Mcap = round_up(n_nodes < 16 ? 16 : n_nodes, 16);
+// A prefill chunk carries as many rows as one pass can (every chunk streams all weights once).
+constexpr int kPrefillRows = kMaxRows;
+
+void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, size_t* kv_bytes, int* Mver_out = nullptr) {
+  const int Mver = round_up(n_nodes < 16 ? 16 : n_nodes, 16);
+  const int Mcap = Mver > kPrefillRows ? Mver : kPrefillRows;
+  if (Mver_out) *Mver_out = Mver;
   const size_t esz = c.weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
   const size_t d = c.d_model, F = c.d_ffn, V = c.vocab, half = c.head_dim / 2;
   Layout l;
@@ -590,8 +596,8 @@ amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_ar
                       ctx->at<int>(l.tok), ctx->at<RowMeta>(l.meta_v), st);
     }
   }
-  target_forward(ctx, ctx->Mcap, ctx->ctx_hi + N);
-  target_head(ctx, ctx->Mcap);
+  target_forward(ctx, ctx->Mver, ctx->ctx_hi + N);
+  target_head(ctx, ctx->Mver);
   return copy_out(ctx, out_argmax, ctx->at<int>(l.amax), sizeof(int) * N);
 }
 
@@ -659,9 +665,9 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   if (!kv_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "kv_dev and ws_dev must not be NULL");
   if (((uintptr_t)kv_dev | (uintptr_t)ws_dev) & 255) return fail(nullptr, AMPH_ERR_WORKSPACE, "regions must be 256-byte aligned");
   Layout l;
-  int Mcap;
+  int Mcap, Mver;
   size_t need_kv;
-  make_layout(*cfg, tree->n_nodes, &l, &Mcap, &need_kv);
+  make_layout(*cfg, tree->n_nodes, &l, &Mcap, &need_kv, &Mver);
   if (kv_bytes < need_kv) return fail(nullptr, AMPH_ERR_WORKSPACE, "kv region: %zu bytes given, %zu needed", kv_bytes, need_kv);
   if (ws_bytes < l.total) return fail(nullptr, AMPH_ERR_WORKSPACE, "workspace: %zu bytes given, %zu needed", ws_bytes, l.total);
   int dev_count = 0;
@@ -676,6 +682,7 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   ctx->dtype = cfg->weight_dtype;
   ctx->esz = cfg->weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
   ctx->Mcap = Mcap;
+  ctx->Mver = Mver;
   ctx->rows_small = 16;
   ctx->lay = l;
   ctx->ws = (char*)ws_dev;
@@ -767,14 +774,15 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
     rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.tok), prompt_ids + start, sizeof(int) * nr, cudaMemcpyHostToDevice, st), "prompt upload");
     if (rc != AMPH_OK) return rc;
     launch_meta_chain(ctx->at<RowMeta>(l.meta_v), start, nr, st);
-    target_forward(ctx, M, start + nr);
-    if (last) target_head(ctx, M);
+    const int rows = round_up(nr, 16);           // rows the kernels carry for this chunk
+    target_forward(ctx, rows, start + nr);
+    if (last) target_head(ctx, rows);
     const int nrs = last ? nr - 1 : nr;           // the last prompt row stays pending for the first draft
     if (nrs > 0 && c.n_sal > 0) {
       rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.next_tok), prompt_ids + start + 1, sizeof(int) * nrs, cudaMemcpyHostToDevice, st), "prompt upload");
       if (rc != AMPH_OK) return rc;
       launch_meta_chain(ctx->at<RowMeta>(l.meta_s), start, nrs, st);
-      run_sals(ctx, ctx->at<float>(l.hidden), ctx->at<int>(l.next_tok), M, start + nrs);
+      run_sals(ctx, ctx->at<float>(l.hidden), ctx->at<int>(l.next_tok), rows, start + nrs);
     }
     if (last)
       launch_prefill_tail(ctx->at<DevState>(l.state), ctx->at<int>(l.amax), nr - 1, ctx->at<float>(l.hidden),
@@ -875,9 +883,9 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
   if (!name || !dst) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and dst must not be NULL");
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
-  const size_t d = c.d_model, V = c.vocab, N = ctx->tree_host.n_nodes, K = c.K;
+  const size_t d = c.d_model, V = c.vocab, N = ctx->tree_host.n_nodes, K = c.K, R = ctx->Mcap;
   struct { const char* n; size_t off, size; } plain[] = {
-      {"hidden", l.hidden, 4 * N * d},   {"logits", l.logits, 4 * N * V},     {"d_logits", l.d_logits, 4 * K * V},
+      {"hidden", l.hidden, 4 * R * d},   {"logits", l.logits, 4 * R * V},     {"d_logits", l.d_logits, 4 * K * V},
       {"hp", l.hp, 4 * K * d},           {"attn_o", l.attn_o, 4 * K * d},     {"sal_h", l.last, 4 * 2 * d},
       {"tree_tokens", l.tok, 4 * N},     {"argmax", l.amax, 4 * N},
   };

@@ -68,7 +68,7 @@ def test_small_bf16_eight_steps(planted, flags):
 
 
 def test_long_prompt_many_attention_splits_fp32():
-    """A 300-token context: several KV splits per head, five prefill chunks (fp32: tight tolerance)."""
+    """A 300-token context: several KV splits per head, three prefill chunks (fp32: tight tolerance)."""
     shape = inputs.get_shape("tiny").with_(prompt_len=300)
     topo = inputs.make_tree(shape.n_nodes, shape.topk)
     model, orc = _setup(shape, topo)
