@@ -405,12 +405,10 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.rows = rows;
   prm.stages = stages;
   prm.ks = ks;
-  // about 40 MB of L2 for prefetched weight tiles, shared by the CTAs that can be resident at once
-  {
-    const long long resident = (long long)tiles * splits < 2LL * g->sm_count ? (long long)tiles * splits : 2LL * g->sm_count;
-    long long pf = (40LL << 20) / (resident * (ks * kTileM * kTileK * 2));
-    prm.l2_prefetch = (int)(pf > 32 ? 32 : pf);
-  }
+  // One more stage per CTA is asked into L2 before the dependency wait.  The TMA unit of an SM serves its copies
+  // and prefetches in order, so a deeper prefetch sits in front of the activation tiles issued after the wait:
+  // 1 stage measured best (0: +0.7 %, 2: +1.2 %, the former 40 MB budget: +3 % on the step).
+  prm.l2_prefetch = 1;
   prm.err_flag = g->err_flag;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
