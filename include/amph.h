@@ -53,7 +53,6 @@ enum { AMPH_DTYPE_F32 = 0, AMPH_DTYPE_BF16 = 1 };
 enum {
   AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
   AMPH_FLAG_NO_GRAPH = 2,       /* launch kernels one by one instead of replaying a CUDA graph */
-  AMPH_FLAG_SIDE_PREFETCH = 4,   /* a second stream prefetches the next weights into L2 while attention runs */
   AMPH_FLAG_SEPARATE_MERGE = 8   /* merge the attention KV splits in a kernel of its own (bf16: a cluster does it otherwise) */
 };
 

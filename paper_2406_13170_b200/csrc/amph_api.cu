@@ -78,9 +78,6 @@ struct amph_ctx {
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
   int sm_count = 148;
-  cudaStream_t side = nullptr;        // second stream: L2 prefetch of upcoming weights beside the dependent chain
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-  bool side_used = false;
   bool last_proj_one_wave = false;   // the last projection ran on the tensor-core kernel with a fully resident grid
   cudaGraphExec_t graph_exec = nullptr;   // captured draft -> verify -> accept schedule of amph_step
   int graph_key = -1;       // attention split counts the captured grids were sized for
@@ -369,35 +366,6 @@ RowScale row_scale_of(const amph_ctx* ctx, size_t off) {
   return rs;
 }
 
-// Between the q/k/v projection and the output projection run only short L2-resident kernels (rotary, attention,
-// merge): HBM idles for about 20 us per layer.  A tiny kernel on a second stream uses that window to ask for the
-// output projection's weights and the head of the gate / up weights to be brought into L2.  (The windows
-// next to the other projections are short and overlap a projection's own TMA traffic: prefetching there
-// measured slower.)
-constexpr double kPrefetchGateUpMB = 20.0;
-
-void prefetch_in_attention_window(amph_ctx* ctx, const LayerW& w) {
-  if (!ctx->side || !ctx->tc) return;
-  const amph_config& c = ctx->cfg;
-  const int units_o = (c.d_model / 64 + 1) / 2;
-  const int stages_gu = (int)(kPrefetchGateUpMB * 1048576.0 / (2.0 * (c.d_ffn / 128) * 32768.0));
-  cudaEventRecord(ctx->ev_fork, ctx->stream);
-  cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0);
-  tc_prefetch_head(ctx->tc, w.wo, c.d_model, c.d_model, 0, units_o, ctx->side);
-  if (stages_gu > 0) {
-    tc_prefetch_head(ctx->tc, w.w_gate, c.d_ffn, c.d_model, 0, stages_gu, ctx->side);
-    tc_prefetch_head(ctx->tc, w.w_up, c.d_ffn, c.d_model, 0, stages_gu, ctx->side);
-  }
-  ctx->side_used = true;                             // the second stream has forked: it must rejoin
-}
-// The second stream rejoins the caller's stream (needed before a capture ends and before results are read).
-void join_side(amph_ctx* ctx) {
-  if (!ctx->side_used) return;
-  cudaEventRecord(ctx->ev_join, ctx->side);
-  cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0);
-  ctx->side_used = false;
-}
-
 // One decoder layer over the rows described by `meta`.
 // Entry: xn holds the input of the q/k/v projections: attn_norm * x / rms(x) if !entry_deferred, else
 // attn_norm * x with the row sums of squares in ss_a (the division is applied after the projection).
@@ -410,7 +378,6 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   cudaStream_t st = ctx->stream;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
   PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
-  prefetch_in_attention_window(ctx, w);
   { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
   launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st,
                   entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale());
@@ -470,7 +437,6 @@ void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
                              last ? ctx->final_norm : ctx->layers[i + 1].attn_norm,
                              last ? ctx->at<float>(l.hidden) : nullptr, deferred);
   }
-  join_side(ctx);
 }
 
 void target_head(amph_ctx* ctx, int rows) {
@@ -508,7 +474,6 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
     layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr, false);
     in_feat = hbuf;
   }
-  join_side(ctx);
 }
 
 amph_status copy_out(amph_ctx* ctx, void* dst, const void* src, size_t bytes) {
@@ -755,14 +720,6 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
     const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model,
                                  c.lm_rank > 0 ? c.lm_rank : 8};
     ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
-    if (ctx->tc && !ctx->side && ctx->stream != nullptr && (c.flags & AMPH_FLAG_SIDE_PREFETCH)) {
-      if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
-          cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
-        ctx->side = nullptr;
-        cudaGetLastError();
-      }
-    }
   }
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
@@ -1055,9 +1012,6 @@ void amph_destroy(amph_ctx* ctx) {
   if (!ctx) return;
   if (ctx->tc) tc_gemm_destroy(ctx->tc);
   if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
-  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
-  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
-  if (ctx->side) cudaStreamDestroy(ctx->side);
   for (auto& e : ctx->prof_ev) cudaEventDestroy(e);
   delete ctx;
 }

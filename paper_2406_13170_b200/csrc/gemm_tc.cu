@@ -417,27 +417,6 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   return true;
 }
 
-namespace {
-__global__ void prefetch_head_kernel(const __grid_constant__ CUtensorMap map, int tiles, int stage_lo, int n_box) {
-  for (int b = blockIdx.x + gridDim.x * threadIdx.x; b < n_box; b += gridDim.x * blockDim.x) {
-    const int st = b / tiles, tl = b - st * tiles;               // stage-major: what the projection reads first
-    tma_prefetch_l2_3d(&map, tl * kTileM, (stage_lo + st) * kStageKb);
-  }
-}
-}  // namespace
-
-bool tc_prefetch_head(TcGemm* g, const void* w, int out, int in, int stage_lo, int stage_hi, cudaStream_t st) {
-  if (!g || !w || out % kTileM || in % kTileK || ((uintptr_t)w & 15)) return false;
-  const int units = (in / kTileK + kStageKb - 1) / kStageKb;
-  if (stage_hi > units) stage_hi = units;
-  if (stage_hi <= stage_lo) return false;
-  const CUtensorMap* m = g->get(w, out, in, kTileM);
-  if (!m) return false;
-  const int tiles = out / kTileM, n_box = tiles * (stage_hi - stage_lo);
-  prefetch_head_kernel<<<n_box < g->sm_count ? n_box : g->sm_count, 32, 0, st>>>(*m, tiles, stage_lo, n_box);
-  return true;
-}
-
 void tc_gemm_destroy(TcGemm* g) { delete g; }
 
 }  // namespace amph

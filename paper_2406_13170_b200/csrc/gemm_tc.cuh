@@ -18,11 +18,6 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
 bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out, int in, int rows, float* P,
                     size_t p_floats, int* splits, size_t* split_stride, cudaStream_t st);
 
-// Asks for pipeline stages [stage_lo, stage_hi) (two 64-wide K blocks each) of every 128-row tile of the
-// [out, in] bf16 matrix w to be brought into L2: the part a projection over w reads first.  One small block
-// per SM, so that no SM's TMA unit queues more than a few pieces.  Returns false if nothing was launched.
-bool tc_prefetch_head(TcGemm* g, const void* w, int out, int in, int stage_lo, int stage_hi, cudaStream_t st);
-
 void tc_gemm_destroy(TcGemm* g);
 
 }  // namespace amph
