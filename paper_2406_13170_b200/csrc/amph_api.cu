@@ -37,7 +37,7 @@ struct Layout {
     return off;
   }
   size_t state, tree, meta_v, meta_s, kv_tab, inv_freq, rope_v, rope_s;
-  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals, topk_cand;
+  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals, topk_cand, amax_cand;
   size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act, lr_act;
   size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
@@ -208,6 +208,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.topk_ids = l.take(sizeof(int) * kMaxK * kTopkStride);
   l.topk_vals = l.take(sizeof(float) * kMaxK * kTopkStride);
   l.topk_cand = l.take(2 * sizeof(float) * kMaxK * kTopkCandChunks * kTopkStride);
+  l.amax_cand = l.take(2 * sizeof(float) * kMaxRows * 8);
   l.x = l.take(4 * Mcap * d);
   l.hidden = l.take(4 * Mcap * d);
   l.h1 = l.take(4 * Mcap * d);
@@ -445,7 +446,7 @@ void target_head(amph_ctx* ctx, int rows) {
   const void* w[1] = {ctx->lm_head};
   PartialView P = project(ctx, XB_XN, w, 1, c.vocab, c.d_model, rows);
   { ProfScope ps(ctx, AMPH_PROF_SELECT);
-  launch_argmax_rows(P, c.vocab, rows, ctx->at<int>(l.amax), ctx->at<float>(l.logits), ctx->stream);
+  launch_argmax_rows(P, c.vocab, rows, ctx->at<int>(l.amax), ctx->at<float>(l.logits), ctx->at<float>(l.amax_cand), ctx->stream);
   }
 }
 

@@ -168,7 +168,8 @@ void launch_gather_diag(PartialView P, void* out_act, int dtype, int K, int r, c
 constexpr int kTopkCandChunks = 32;
 void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids, float* vals,
                        float* d_logits, float* cand, cudaStream_t st);
-void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st);
+// cand: scratch for the slices' candidates, kMaxRows * 8 (value, id) pairs
+void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, float* cand, cudaStream_t st);
 
 // ---- control kernels
 void launch_meta_chain(RowMeta* meta, int base, int n_rows, cudaStream_t st);             // prefill chunk

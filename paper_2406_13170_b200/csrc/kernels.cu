@@ -862,26 +862,63 @@ void launch_topk_heads(PartialView P, int vocab, int K, const int* ck, int* ids,
   launch_pdl(topk_merge_kernel, dim3(K), dim3(kTopkThreads), 0, st, reinterpret_cast<const float2*>(cand), n_chunks, c, ids, vals);
 }
 
-__global__ void argmax_rows_kernel(PartialView P, int vocab, int* __restrict__ amax,
-                                   float* __restrict__ logits_out) {
+// Greedy choice per verified row in two stages, like the top-k above: block (row, slice) reduces the partials of
+// its slice of the row, stores the logits (debug tap) and its best (value, id); one thread per row then merges the
+// slices (ties -> lowest id, the same order as a single pass).
+constexpr int kArgmaxSlices = 8;
+
+__global__ void __launch_bounds__(256)
+argmax_slice_kernel(PartialView P, int vocab, int chunk, float2* __restrict__ cand, float* __restrict__ logits_out, int vec) {
   pdl_wait();
   pdl_launch_dependents();
   __shared__ float sv[32];
   __shared__ int si[32];
-  const int r = blockIdx.x;
+  const int r = blockIdx.x, j = blockIdx.y;
+  const int lo = j * chunk, hi = lo + chunk < vocab ? lo + chunk : vocab;
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
-    const float v = sum_partials(P, r, c);
-    if (logits_out) logits_out[(size_t)r * vocab + c] = v;
-    if (better(v, c, bv, bi)) { bv = v; bi = c; }
+  for (int c = lo + threadIdx.x * 4; c < hi; c += blockDim.x * 4) {
+    if (vec && c + 3 < hi) {
+      const float4 v = sum_partials4(P, r, c);
+      if (logits_out) store4(logits_out + (size_t)r * vocab + c, v);
+      if (better(v.x, c, bv, bi)) { bv = v.x; bi = c; }
+      if (better(v.y, c + 1, bv, bi)) { bv = v.y; bi = c + 1; }
+      if (better(v.z, c + 2, bv, bi)) { bv = v.z; bi = c + 2; }
+      if (better(v.w, c + 3, bv, bi)) { bv = v.w; bi = c + 3; }
+    } else {
+      for (int e = c; e < hi && e < c + 4; ++e) {
+        const float v = sum_partials(P, r, e);
+        if (logits_out) logits_out[(size_t)r * vocab + e] = v;
+        if (better(v, e, bv, bi)) { bv = v; bi = e; }
+      }
+    }
   }
   block_best(bv, bi, sv, si);
-  if (threadIdx.x == 0) amax[r] = bi;
+  if (threadIdx.x == 0) cand[r * kArgmaxSlices + j] = make_float2(bv, __int_as_float(bi));
 }
 
-void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, cudaStream_t st) {
-  launch_pdl(argmax_rows_kernel, dim3(rows), dim3(1024), 0, st, P, vocab, amax, logits_out);
+__global__ void argmax_merge_kernel(const float2* __restrict__ cand, int n_slices, int rows, int* __restrict__ amax) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int j = 0; j < n_slices; ++j) {
+    const float2 e = cand[r * kArgmaxSlices + j];
+    const int id = __float_as_int(e.y);
+    if (better(e.x, id, bv, bi)) { bv = e.x; bi = id; }
+  }
+  amax[r] = bi;
+}
+
+void launch_argmax_rows(PartialView P, int vocab, int rows, int* amax, float* logits_out, float* cand, cudaStream_t st) {
+  const int vec = vocab % 4 == 0 && P.ld % 4 == 0;
+  int chunk = (vocab + kArgmaxSlices - 1) / kArgmaxSlices;
+  chunk = (chunk + 3) / 4 * 4;
+  const int n_slices = (vocab + chunk - 1) / chunk;
+  launch_pdl(argmax_slice_kernel, dim3(rows, n_slices), dim3(256), 0, st, P, vocab, chunk, reinterpret_cast<float2*>(cand), logits_out, vec);
+  launch_pdl(argmax_merge_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, reinterpret_cast<const float2*>(cand), n_slices, rows, amax);
 }
 
 // --------------------------------------------------------------------------------------------
