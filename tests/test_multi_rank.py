@@ -56,3 +56,15 @@ def test_reference_arm_other_ranks_exit_without_work():
                         "--steps", "1", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0
     assert r.stdout.strip() == ""
+
+
+def test_roofline_traffic_is_null_once_the_kernel_source_changed(monkeypatch):
+    """`roofline.traffic` comes from one ncu capture of one version of the projection kernel: it is reported only
+    while the kernel's source still has the digest recorded with the capture."""
+    sys.path.insert(0, ROOT)
+    import bench
+    monkeypatch.setattr(bench, "NCU_KERNEL_SOURCE_SHA256_16", "0" * 16)
+    assert bench.ncu_traffic(1.0e8) is None
+    monkeypatch.undo()
+    t = bench.ncu_traffic(1.0e8)
+    assert t is None or 1.0e8 <= t <= 1.1e8          # traffic = weight bytes plus the partial sums, no re-reads
