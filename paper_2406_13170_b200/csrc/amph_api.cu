@@ -395,10 +395,19 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st,
                      ctx->last_proj_one_wave);
   }
-  const void* gu[2] = {w.w_gate, w.w_up};
-  P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
-  { ProfScope ps(ctx, AMPH_PROF_SWIGLU);
-  launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b), ctx->last_proj_one_wave);
+  bool fused_gu = false;
+  if (ctx->tc && !(c.flags & AMPH_FLAG_SEPARATE_SWIGLU)) {         // gate / up projection with SwiGLU in its epilogue
+    ProfScope ps(ctx, AMPH_PROF_PROJECTION);
+    fused_gu = tc_gemm_launch_swiglu(ctx->tc, XB_XN, w.w_gate, w.w_up, c.d_ffn, c.d_model, rows, ctx->ws + l.act,
+                                     row_scale_of(ctx, l.ss_b), st);
+    if (fused_gu && ps.rec) ctx->prof_bytes += 2LL * c.d_ffn * c.d_model * (int64_t)ctx->esz;
+    if (fused_gu) ctx->last_proj_one_wave = false;
+  }
+  if (!fused_gu) {
+    const void* gu[2] = {w.w_gate, w.w_up};
+    P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
+    ProfScope ps(ctx, AMPH_PROF_SWIGLU);
+    launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b), ctx->last_proj_one_wave);
   }
   const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);

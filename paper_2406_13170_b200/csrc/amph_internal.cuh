@@ -101,6 +101,27 @@ struct RowScale {
 };
 constexpr int kScaleChunkCols = 512;     // columns per block of resid_scale_kernel (128 threads x float4)
 
+#ifdef __CUDACC__
+// value(row, col .. col+3) of a projection left as split-K partial sums (fixed order: deterministic)
+__device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, int col) {
+  const float* p = P.p + (size_t)row * P.ld + col;
+  float4 acc = *reinterpret_cast<const float4*>(p);
+#pragma unroll 4
+  for (int s = 1; s < P.splits; ++s) {
+    const float4 v = *reinterpret_cast<const float4*>(p + (size_t)s * P.split_stride);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  return acc;
+}
+__device__ __forceinline__ float row_scale(const RowScale& rs, int row) {
+  if (rs.ss == nullptr) return 1.0f;
+  float tot = 0.f;
+#pragma unroll 8
+  for (int c = 0; c < rs.chunks; ++c) tot += rs.ss[row * rs.chunks + c];       // fixed order
+  return 1.0f / sqrtf(tot / (float)rs.d + rs.eps);
+}
+#endif
+
 // ---- launchers (one per kernel family); dtype = AMPH_DTYPE_* of weights / activations / cache
 void launch_embed(const void* tok_emb, int dtype, const int* toks, int vocab, int rows, int d,
                   float* x, cudaStream_t st);

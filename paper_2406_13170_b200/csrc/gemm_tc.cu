@@ -48,6 +48,12 @@ struct TcParams {
   int stages;
   int l2_prefetch;          // weight tiles (beyond the ring) each CTA pulls into L2 before it waits
   int ks;                   // K blocks per stage (depth of the tensor maps' boxes): kStageKb, or 1 for many activation rows
+  // SWIGLU launches: a tile is 64 gate rows + the 64 up rows of the same features; the epilogue writes
+  //   act[row][feature] = silu(gate * inv_rms(row)) * (up * inv_rms(row))   (bf16, row pitch f)
+  __nv_bfloat16* act;
+  int f;
+  int up_first;             // the tensor map's outer index 0 is the up matrix (it has the lower address)
+  RowScale rs;
   int* err_flag;
 };
 
@@ -111,6 +117,18 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int r
   asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(0), "r"(row), "r"(kb) : "memory");
 }
 
+// 4-D form for the fused gate / up launch: (column, row, K block, matrix) with the distance between the two weight
+// matrices as the outermost stride, so ONE copy brings the gate and the up rows of a tile.
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(0), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int row, int kb) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(0), "r"(row), "r"(kb), "r"(0) : "memory");
+}
+
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -129,9 +147,9 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   return d;
 }
 
-// Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = nt.
-__device__ __forceinline__ uint32_t umma_idesc(int nt) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, M = m (128 or 64), N = nt.
+__device__ __forceinline__ uint32_t umma_idesc(int nt, int m = kTileM) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
@@ -146,9 +164,15 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// SWIGLU: the gate / up projection with SwiGLU in the epilogue.  A CTA owns 64 features and the whole K range; per K
+// step it issues two M = 64 MMAs, gate rows into accumulator columns [0, nt) and up rows into [ntc, ntc + nt).  Row r
+// of an M = 64 accumulator lives in TMEM lane 32 (r / 16) + r % 16 (checked on the device), so lane l < 16 of the
+// epilogue warp of quarter q holds gate and up of feature 16 q + l for all rows: no exchange between warps.
+template <bool SWIGLU>
 __global__ void __launch_bounds__(kThreads)
 tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ float inv_s[SWIGLU ? kTileM : 1];         // 1 / rms of the activation rows (SWIGLU)
   __shared__ __align__(8) uint64_t full_bar[8];
   __shared__ __align__(8) uint64_t empty_bar[8];
   __shared__ __align__(8) uint64_t accum_bar;
@@ -159,7 +183,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
-  const int row0 = (tile - seg * prm.tiles_per_seg) * kTileM;       // first weight row of this tile
+  const int row0 = SWIGLU ? tile * (kTileM / 2) : (tile - seg * prm.tiles_per_seg) * kTileM;   // first weight row of this tile
   // K range of this split in whole stages (ks blocks), so that every copy starts on a stage boundary
   const int ks = prm.ks;
   const int units = (prm.kblocks + ks - 1) / ks;
@@ -173,8 +197,9 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const uint32_t a_bytes = ks * a_tile, b_bytes = ks * b_tile;
   const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < nt) tmem_cols <<= 1;
+  uint32_t ntc = 32;
+  while ((int)ntc < nt) ntc <<= 1;
+  const uint32_t tmem_cols = SWIGLU ? 2 * ntc : ntc;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -206,10 +231,14 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     if (leader) {
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
-        tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
+        if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
+        else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
-      for (int i = npre; i < npf; ++i) tma_prefetch_l2_3d(wmap, row0, kb_lo + i * ks);
+      for (int i = npre; i < npf; ++i) {
+        if (SWIGLU) tma_prefetch_l2_4d(wmap, row0, kb_lo + i * ks);
+        else tma_prefetch_l2_3d(wmap, row0, kb_lo + i * ks);
+      }
     }
     __syncwarp();
     pdl_wait();
@@ -224,7 +253,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
+        if (SWIGLU) tma_load_4d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
+        else tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
         tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[s]);
       }
       __syncwarp();
@@ -241,7 +271,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   } else if (warp == 1) {
     // ---------------- MMA issuer (the warp stays converged, its elected lane issues)
     const bool leader = elect_one();
-    const uint32_t idesc = umma_idesc(nt);
+    const uint32_t idesc = umma_idesc(nt, SWIGLU ? kTileM / 2 : kTileM);
     bool ok = true;
     for (int i = 0; i < nit; ++i) {
       const int s = i % stages, round = i / stages;
@@ -252,10 +282,24 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
         const int nk = nkb - i * ks < ks ? nkb - i * ks : ks;   // blocks of the stage inside the K range
         for (int kk = 0; kk < nk; ++kk) {
-          const uint64_t adesc = umma_desc(a_addr + (uint32_t)kk * a_tile), bdesc = umma_desc(a_addr + a_bytes + (uint32_t)kk * b_tile);
+          const uint64_t bdesc = umma_desc(a_addr + a_bytes + (uint32_t)kk * b_tile);
+          if constexpr (SWIGLU) {
+            // the copy landed as [matrix][K block][64 rows]: two half tiles per K block, one MMA each
+            const uint32_t half = a_tile / 2;
+            const int gi = prm.up_first ? 1 : 0;
+            const uint64_t gdesc = umma_desc(a_addr + (uint32_t)(gi * ks + kk) * half);
+            const uint64_t udesc = umma_desc(a_addr + (uint32_t)((1 - gi) * ks + kk) * half);
 #pragma unroll
-          for (int k = 0; k < kTileK / kUmmaK; ++k)    // +32 bytes (2 x 16 B) per K step inside the swizzle row
-            umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+            for (int k = 0; k < kTileK / kUmmaK; ++k) {
+              umma_f16(tmem_d, gdesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+              umma_f16(tmem_d + ntc, udesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+            }
+          } else {
+            const uint64_t adesc = umma_desc(a_addr + (uint32_t)kk * a_tile);
+#pragma unroll
+            for (int k = 0; k < kTileK / kUmmaK; ++k)    // +32 bytes (2 x 16 B) per K step inside the swizzle row
+              umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+          }
         }
         umma_commit(&empty_bar[s]);                    // frees the stage once these MMAs have read it
       }
@@ -267,8 +311,57 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
     const int quarter = warp & 3;
     pdl_wait();                                      // P may still be read by the kernel before this one
+    if constexpr (SWIGLU) {                          // 1 / rms of the rows, while the main loop runs
+      const int et = threadIdx.x - 64;
+      if (et < prm.rows) inv_s[et] = row_scale(prm.rs, et);
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
     const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag) : false);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if constexpr (SWIGLU) {
+      // lanes 0..15 of the warp of quarter q hold features 16 q .. 16 q + 15 of the tile (gate and up alike); the
+      // upper half of the warp takes over the second half of each block of 16 rows
+      const int feat = row0 + quarter * 16 + (lane & 15);
+      const int jb = (lane >> 4) * 8;
+      for (int c0 = 0; c0 < nt && c0 < prm.rows; c0 += 16) {
+        uint32_t g[16], u[16];
+        const uint32_t taddr = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
+        if (ok) {
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+              : "=r"(g[0]), "=r"(g[1]), "=r"(g[2]), "=r"(g[3]), "=r"(g[4]), "=r"(g[5]), "=r"(g[6]), "=r"(g[7]),
+                "=r"(g[8]), "=r"(g[9]), "=r"(g[10]), "=r"(g[11]), "=r"(g[12]), "=r"(g[13]), "=r"(g[14]), "=r"(g[15])
+              : "r"(taddr)
+              : "memory");
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+              : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+              : "r"(taddr + ntc)
+              : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) g[j] = u[j] = 0u;
+        }
+        float gv[8], uv[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {                  // rows c0 + 8 .. c0 + 15 move to lanes 16 .. 31
+          const uint32_t gh = __shfl_sync(0xffffffffu, g[8 + j], lane & 15), uh = __shfl_sync(0xffffffffu, u[8 + j], lane & 15);
+          gv[j] = __uint_as_float(lane < 16 ? g[j] : gh);
+          uv[j] = __uint_as_float(lane < 16 ? u[j] : uh);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = c0 + jb + j;
+          if (r < prm.rows) {
+            const float sc = inv_s[r];
+            const float t = gv[j] * sc;
+            prm.act[(size_t)r * prm.f + feat] = __float2bfloat16(__fdividef(t, 1.0f + __expf(-t)) * (uv[j] * sc));
+          }
+        }
+      }
+    } else {
     const int feat = seg * prm.tiles_per_seg * kTileM + row0 + quarter * 32 + lane;
     float* out = prm.P + (size_t)split * prm.split_stride + feat;
     for (int c0 = 0; c0 < nt; c0 += 16) {
@@ -290,6 +383,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
 #pragma unroll
       for (int j = 0; j < 16; ++j)
         if (c0 + j < prm.rows) out[(size_t)(c0 + j) * prm.ld] = __uint_as_float(v[j]);
+    }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -316,6 +410,26 @@ struct TcGemm {
   std::map<std::tuple<const void*, int, int, int, int>, CUtensorMap> cache;   // (ptr, rows, cols, box rows, box K blocks)
   int sm_count = 148;
   int max_smem = 0;
+  std::map<std::tuple<const void*, const void*, int, int, int>, CUtensorMap> pair_cache;   // (lower, upper matrix, rows, cols, K blocks)
+
+  // Two [rows, cols] matrices as one 4-D tensor (column, row, K block, matrix): a box of 64 rows of both.
+  const CUtensorMap* get_pair(const void* lo, const void* hi, int rows, int cols, int box_kb) {
+    auto key = std::make_tuple(lo, hi, rows, cols, box_kb);
+    auto it = pair_cache.find(key);
+    if (it != pair_cache.end()) return &it->second;
+    const uint64_t gap = (uint64_t)((const char*)hi - (const char*)lo);
+    if (gap == 0 || (gap & 15) || gap >= (1ull << 40)) return nullptr;
+    CUtensorMap m;
+    const cuuint64_t dims[4] = {(cuuint64_t)kTileK, (cuuint64_t)rows, (cuuint64_t)cols / kTileK, 2};
+    const cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)kTileK * 2, (cuuint64_t)gap};
+    const cuuint32_t box[4] = {(cuuint32_t)kTileK, (cuuint32_t)(kTileM / 2), (cuuint32_t)box_kb, 2};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(lo), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return nullptr;
+    return &(pair_cache[key] = m);
+  }
 
   const CUtensorMap* get(const void* ptr, int rows, int cols, int box_rows, int box_kb = kStageKb) {
     auto key = std::make_tuple(ptr, rows, cols, box_rows, box_kb);
@@ -355,7 +469,8 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
   for (int i = 0; i < n; ++i) { g->xptr[i] = xbufs[i]; g->xrows[i] = xrows[i]; g->xcols[i] = xcols[i]; }
   cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&g->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
   return g;
 }
 
@@ -411,10 +526,49 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.l2_prefetch = 1;
   prm.err_flag = g->err_flag;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  launch_pdl(tc_gemm_kernel, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
+  launch_pdl(tc_gemm_kernel<false>, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
   *split_stride = prm.split_stride;
   return true;
+}
+
+bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_up, int f, int in, int rows, void* act,
+                           const RowScale& rs, cudaStream_t st) {
+  if (!g || xb < 0 || xb >= g->n_x || !w_gate || !w_up || !act) return false;
+  if (f % (kTileM / 2) || in % kTileK || rows < 1 || g->xcols[xb] != in) return false;
+  if (((uintptr_t)w_gate | (uintptr_t)w_up) & 15) return false;
+  const int nt = rows <= 16 ? 16 : (rows + 15) / 16 * 16;
+  if (nt > 64 || nt > g->xrows[xb]) return false;          // two accumulators of nt columns; stages of two K blocks
+  const int ks = kStageKb, kblocks = in / kTileK, tiles = f / (kTileM / 2);
+  const bool up_first = (const char*)w_up < (const char*)w_gate;
+  const CUtensorMap* mw = g->get_pair(up_first ? w_up : w_gate, up_first ? w_gate : w_up, f, in, ks);
+  const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt, ks);
+  if (!mw || !mx) return false;
+  TmapPack pack;
+  memset(&pack, 0, sizeof pack);
+  pack.w[0] = *mw;
+  pack.x = *mx;
+  const uint32_t stage_bytes = ks * kTileM * kTileK * 2 + ((ks * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  int stages = (int)((110 * 1024) / stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  TcParams prm;
+  memset(&prm, 0, sizeof prm);
+  prm.tiles_per_seg = tiles;
+  prm.kblocks = kblocks;
+  prm.splits = 1;
+  prm.nt = nt;
+  prm.rows = rows;
+  prm.stages = stages;
+  prm.ks = ks;
+  prm.l2_prefetch = 1;
+  prm.act = (__nv_bfloat16*)act;
+  prm.f = f;
+  prm.up_first = up_first ? 1 : 0;
+  prm.rs = rs;
+  prm.err_flag = g->err_flag;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  return launch_pdl(tc_gemm_kernel<true>, dim3(tiles, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
 }
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }

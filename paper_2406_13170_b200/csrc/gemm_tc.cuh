@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 
+#include "amph_internal.cuh"
+
 namespace amph {
 
 struct TcGemm;
@@ -17,6 +19,13 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
 // Returns false (nothing launched) if the shape is not covered; the caller then uses the plain kernel.
 bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out, int in, int rows, float* P,
                     size_t p_floats, int* splits, size_t* split_stride, cudaStream_t st);
+
+// Gate / up projection with SwiGLU in the epilogue (no partial sums, no separate kernel):
+//   act[row][o] = silu(g * s) * (u * s),  g = X[row] . W_gate[o],  u = X[row] . W_up[o],  s = the row's deferred RMSNorm scale.
+// w_gate, w_up: bf16 [f, in]; act: bf16 [rows][f].  Takes at most 64 rows and needs the two matrices less than 1 TB
+// apart (they are fetched through one tensor map); returns false, nothing launched, if the form is not available.
+bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_up, int f, int in, int rows, void* act,
+                           const RowScale& rs, cudaStream_t st);
 
 void tc_gemm_destroy(TcGemm* g);
 

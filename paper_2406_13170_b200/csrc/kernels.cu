@@ -41,16 +41,6 @@ __device__ __forceinline__ void add_splits(const float* p, size_t stride, int s0
     if (s0 + s < splits) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
 }
 
-__device__ __forceinline__ float4 sum_partials4(const PartialView& P, int row, int col) {
-  const float* p = P.p + (size_t)row * P.ld + col;
-  float4 acc = *reinterpret_cast<const float4*>(p);
-#pragma unroll 4
-  for (int s = 1; s < P.splits; ++s) {
-    const float4 v = *reinterpret_cast<const float4*>(p + (size_t)s * P.split_stride);
-    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-  }
-  return acc;
-}
 // Same sum for kernels with registers to spare and many splits to read (the residual kernels).
 __device__ __forceinline__ float4 sum_partials4_wide(const PartialView& P, int row, int col) {
   const float* p = P.p + (size_t)row * P.ld + col;
@@ -74,14 +64,6 @@ __device__ __forceinline__ float4 load4(const bf16* p) {
   const uint2 u = *reinterpret_cast<const uint2*>(p);
   return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
                      __uint_as_float(u.y & 0xffff0000u));
-}
-
-__device__ __forceinline__ float row_scale(const RowScale& rs, int row) {
-  if (rs.ss == nullptr) return 1.0f;
-  float tot = 0.f;
-#pragma unroll 8
-  for (int c = 0; c < rs.chunks; ++c) tot += rs.ss[row * rs.chunks + c];       // fixed order
-  return 1.0f / sqrtf(tot / (float)rs.d + rs.eps);
 }
 
 __device__ __forceinline__ float block_sum(float v, float* red) {

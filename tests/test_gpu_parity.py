@@ -50,7 +50,7 @@ def test_tiny_depth4_tree_and_ragged_prompt():
     model.close()
 
 
-@pytest.mark.parametrize("flags", [1, 0, 8], ids=["plain-kernels", "tensor-core", "separate-merge"])
+@pytest.mark.parametrize("flags", [1, 0, 8, 16], ids=["plain-kernels", "tensor-core", "separate-merge", "separate-swiglu"])
 @pytest.mark.parametrize("planted", [False, True], ids=["natural", "planted"])
 def test_small_bf16_eight_steps(planted, flags):
     """bf16 storage, several 128-row weight tiles, a 32-node tree, a prompt that is not a
