@@ -7,6 +7,7 @@ the benchmark build inputs here and hand the same tensors to both sides.
 from .configs import ModelShape, SHAPES, get_shape  # noqa: F401
 from .gen import (  # noqa: F401
     normal_tensor,
+    tensor_std,
     uniform_ids,
     weight_specs,
     make_weights,

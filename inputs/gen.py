@@ -156,18 +156,32 @@ def weight_specs(shape: ModelShape) -> List[Tuple[str, Tuple[int, ...], str]]:
     return specs
 
 
+def tensor_std(name: str, shp: Tuple[int, ...], std: float, init: str) -> float:
+    """Standard deviation of one tensor.  init "normal": `std` for every tensor (the benchmark's N(0, 0.02)).
+    init "fan_in": every linear map gets 1 / sqrt(in_features), so that it neither amplifies nor damps its
+    input whatever the width (embedding rows have unit variance; biases and position embeddings 0.5)."""
+    if init == "normal":
+        return std
+    if name == "tok_emb":
+        return 1.0
+    if len(shp) == 1 or name == "draft.pe":
+        return 0.5
+    return 1.0 / math.sqrt(shp[-1])
+
+
 def make_weights(shape: ModelShape, seed: int = 0, device="cpu", std: float = 0.02,
-                 only=None) -> Dict[str, torch.Tensor]:
-    """All weights of `shape`: N(0, std) in the shape's storage dtype; norm gains 1."""
+                 only=None, init: str = "normal") -> Dict[str, torch.Tensor]:
+    """All weights of `shape` in its storage dtype; norm gains 1; the rest normal (see tensor_std)."""
+    assert init in ("normal", "fan_in")
     dtype = torch.float32 if shape.dtype == "fp32" else torch.bfloat16
     out: Dict[str, torch.Tensor] = {}
-    for name, shp, init in weight_specs(shape):
+    for name, shp, kind in weight_specs(shape):
         if only is not None and not only(name):
             continue
-        if init == "ones":
+        if kind == "ones":
             out[name] = torch.ones(shp, dtype=dtype, device=device)
         else:
-            out[name] = normal_tensor(shp, std, seed, name, dtype=dtype, device=device)
+            out[name] = normal_tensor(shp, tensor_std(name, shp, std, init), seed, name, dtype=dtype, device=device)
     return out
 
 

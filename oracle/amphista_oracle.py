@@ -22,6 +22,8 @@ Parity status of the parts
     autoregressive decoding, Fig. 5's node / candidate counts, exhaustive
     acceptance patterns, chain-tree == causal forward, single-key attention,
     RoPE relative-position property, torch's own attention routine).
+  * input of the adaptation layers (Eq. 1): concatenation order [hidden ; embedding],
+    which token's embedding, and causality over the pending rows are pinned.
   * draft-module numerics (inside of the adaptation layers, the head MLP form, the
     residual in the Auto-embedding Block): the paper prints no values and ships
     no weights, so beyond the structural pins (permutation equivariance of the

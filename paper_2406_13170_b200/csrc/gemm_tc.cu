@@ -119,10 +119,18 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int r
 
 // 4-D form for the fused gate / up launch: (column, row, K block, matrix) with the distance between the two weight
 // matrices as the outermost stride, so ONE copy brings the gate and the up rows of a tile.
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar) {
+// Weight tiles are read exactly once per pass: they are loaded with an evict-first L2 policy so that the stream of
+// weights (100-180 MB per launch, about the size of L2) does not push out the activations, partial sums and KV rows
+// that the neighbouring kernels re-read from L2 (measured: -3.8 % on the 7B step).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(0), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(0), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int row, int kb) {
@@ -133,6 +141,12 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
 
@@ -219,6 +233,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   if (warp == 0) {
     // ---------------- TMA producer (the warp stays converged, its elected lane issues)
     const bool leader = elect_one();
+    const uint64_t wpol = l2_evict_first_policy();
     const CUtensorMap* wmap = &maps.w[seg];
     if (leader) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(wmap) : "memory");
@@ -231,8 +246,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     if (leader) {
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
-        if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
-        else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i]);
+        if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
+        else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
       for (int i = npre; i < npf; ++i) {
@@ -253,8 +268,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        if (SWIGLU) tma_load_4d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
-        else tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s]);
+        if (SWIGLU) tma_load_4d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
+        else tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
         tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[s]);
       }
       __syncwarp();

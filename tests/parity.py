@@ -26,6 +26,7 @@ class Report:
     max_dlogit_err: float = 0.0
     max_draft_err: float = 0.0
     max_kv_err: float = 0.0
+    own_tree_steps: int = 0        # steps verified on the tree the GPU built from its own candidates
     topk_tie_swaps: int = 0
     argmax_near_ties: int = 0
     gated_steps: int = 0
@@ -127,9 +128,19 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
         # measured error of the draft logits (itself bounded by tol above), or than the stated tie width
         e_abs = float((g_dl.to(torch.float64).cpu() - taps["d_logits"].to(torch.float64)).abs().max())
         compare_topk(shape, g_ids, g_vals, taps["d_logits"], max(tie_tol * scale, 2.0 * e_abs), rep)
-        # ---- verify the oracle's tree tokens
-        toks = torch.tensor(taps["toks"], dtype=torch.int32, device=dev)
-        model.verify_tree(toks, g_amax)
+        # ---- tree construction (Appendix A.1): node 0 carries the root, a depth-k node head k's candidate of its
+        # rank.  The tokens the library gathered must be that function of the library's OWN candidate lists.
+        root_i = int(taps["toks"][0])
+        g_tt = model.get_tensor("tree_tokens", (N,), torch.int32).tolist()
+        assert g_tt == ao.Oracle.tree_tokens(root_i, g_ids.tolist(), t), f"step {i}: tree tokens are not the gathered candidates"
+        # ---- verify.  When the library drafted the oracle's candidates (no near-tie swap) it verifies its own tree:
+        # NULL keeps every drafted token, a planted path arrives as overrides with -1 = "keep the drafted token".
+        # Otherwise both sides verify the oracle's tokens so that the rows stay comparable.
+        if g_tt == ao.Oracle.tree_tokens(root_i, taps["topk_ids"], t):
+            rep.own_tree_steps += 1
+            model.verify_tree(None if ov is None else torch.tensor(ov, dtype=torch.int32, device=dev), g_amax)
+        else:
+            model.verify_tree(torch.tensor(taps["toks"], dtype=torch.int32, device=dev), g_amax)
         torch.cuda.synchronize(dev)
         assert model.get_tensor("tree_tokens", (N,), torch.int32).tolist() == taps["toks"]
         g_logits = model.get_tensor("logits", (N, V))

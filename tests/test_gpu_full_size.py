@@ -1,10 +1,17 @@
 """Parity at the benchmark's full size and at the other large shapes.
 
-The 7B-shape test runs the exact configuration bench.py times (32 layers, d = 4096, vocab 32000, 64-node
-tree, 512-token prompt, tensor-core projections, CUDA-graph step) and compares it with the float32 CPU
-oracle on the same seeded weights: root token, draft logits and candidates, all 64 verified rows, acceptance
-and the compacted cache, for one natural and one planted step.  The 13B / 33B shapes are checked at two
-layers of depth (their widths, head counts and tile counts are what differs from 7B).
+Two kinds of weights are used, both from the same seeded generator:
+  * "fan_in": every linear map has standard deviation 1 / sqrt(in_features), so no layer amplifies its input.
+    On these well-conditioned models the stated tolerance (2e-2 against the plain float32 oracle, which keeps
+    every activation in float32) must hold for the target AND for every tensor of the draft module, at the full
+    depth of the 7B shape (32 layers, the exact launch configuration bench.py times) and at 13B / 33B widths.
+    This is the gate that shows the kernels right at full size (measured: 7e-3 .. 8e-3 at 7B full depth).
+  * "normal": the benchmark's N(0, 0.02) weights.  There every linear map of width d has gain 0.02 * sqrt(d)
+    (1.28 at 4096), the 32-layer stack is ill-conditioned and the rounding of the bf16 storage points grows like
+    a random walk over the layers (measured 4.6e-2 on the target, 0.33 on the draft module's un-normalised
+    vocabulary logits; the oracle's own bf16-storage mode is 3.2e-2 / 0.17 away from the GPU and about as far
+    from the plain oracle).  The run is kept because it is the benchmark's model; its bounds follow the depth
+    and are not the stated tolerance.
 """
 import pytest
 import torch
@@ -34,24 +41,27 @@ def tol_draft(n_layers: int) -> float:
     map of width d has gain 0.02 * sqrt(d) (1.28 at 4096, 1.63 at 6656), so these random-init stacks amplify
     the bf16 storage rounding strongly: measured against the plain oracle 6e-2 .. 0.12 (7B widths, 2-layer
     target), 0.24 (33B widths, 2 layers), 0.25 .. 0.40 (7B, 32 layers).  At these widths closeness of the draft
-    tensors is therefore only bounded loosely (0.6; unrelated outputs give about 1.4); the draft module's
-    arithmetic is pinned tightly by the small-shape tests (1e-5 in fp32, 2e-2 in bf16)."""
-    return 0.6
+    tensors is therefore only bounded loosely here (0.5; unrelated outputs give about 1.4); the stated 2e-2 is
+    shown for the same tensors, at the same sizes, by the well-conditioned twins of these tests."""
+    return 0.5
 
 
-def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1), storage=None):
+def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1), storage=None, init="normal"):
     from paper_2406_13170_b200 import Amphista
     topo = inputs.make_tree(shape.n_nodes, shape.topk)
-    w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0")
+    w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0", init=init)
     w_cpu = {k: v.cpu() for k, v in w_gpu.items()}                 # same generator; device independence is tested elsewhere
-    probe = inputs.normal_tensor(w_cpu["layers.0.wq"].shape, 0.02, 0, "layers.0.wq", dtype=torch.bfloat16)
-    assert torch.equal(probe, w_cpu["layers.0.wq"])
+    wq = w_cpu["layers.0.wq"]
+    probe = inputs.normal_tensor(wq.shape, inputs.tensor_std("layers.0.wq", wq.shape, 0.02, init), 0, "layers.0.wq",
+                                 dtype=torch.bfloat16)
+    assert torch.equal(probe, wq)
     model = Amphista(shape, topo, w_gpu)
     orc = ao.Oracle(shape, w_cpu, dtype=torch.float32, storage=storage)
-    tol = tol_plain(shape.n_layers)
+    well = init == "fan_in"
+    tol = TOL_BF16 if well else tol_plain(shape.n_layers)
     prompt = inputs.make_prompt(shape, n=prompt_len or shape.prompt_len).tolist()
     rep = run_parity(model, orc, shape, topo, prompt, steps, tol, TIE_BF16, planted, kv_check_layers=kv_layers,
-                     tol_draft=tol_draft(shape.n_layers))
+                     tol_draft=TOL_BF16 if well else tol_draft(shape.n_layers))
     print(shape.name, rep)
     # the same context must also run through amph_step (graph replay) and stay consistent with its own state
     out_tok = torch.zeros(shape.K + 1, dtype=torch.int32, device="cuda:0")
@@ -66,15 +76,36 @@ def _run(shape, steps, planted, prompt_len=None, kv_layers=(0, -1), storage=None
     return rep
 
 
-def test_7b_shape_full_depth():
+def test_7b_shape_full_depth_stated_tolerance():
+    """The benchmark's configuration on well-conditioned weights: 2e-2 for target and draft module alike."""
+    shape = inputs.get_shape("7b")
+    rep = _run(shape, 2, True, init="fan_in")
+    assert rep.steps == 2 and max(rep.accepted) >= 2
+    assert max(rep.max_logit_err, rep.max_hidden_err, rep.max_dlogit_err, rep.max_draft_err, rep.max_kv_err) <= TOL_BF16
+
+
+def test_7b_shape_full_depth_benchmark_weights():
+    """The same run on the benchmark's own N(0, 0.02) weights (depth-derived bounds, see the module docstring)."""
     shape = inputs.get_shape("7b")
     rep = _run(shape, 2, True)
     assert rep.steps == 2 and max(rep.accepted) >= 2
 
 
-@pytest.mark.parametrize("storage", [None, torch.bfloat16], ids=["plain-oracle", "bf16-storage-oracle"])
 @pytest.mark.parametrize("name", ["7b", "13b", "33b"])
-def test_large_shapes_two_layers(name, storage):
+def test_large_shapes_two_layers_stated_tolerance(name):
+    """Widths, head counts and tile counts of the three shapes on well-conditioned weights: 2e-2 everywhere."""
     shape = inputs.get_shape(name).with_(n_layers=2, prompt_len=70)
-    rep = _run(shape, 2, True, kv_layers=(0, 1), storage=storage)
+    rep = _run(shape, 2, True, kv_layers=(0, 1), init="fan_in")
     assert rep.steps == 2
+    assert max(rep.max_logit_err, rep.max_hidden_err, rep.max_dlogit_err, rep.max_draft_err, rep.max_kv_err) <= TOL_BF16
+
+
+@pytest.mark.parametrize("name", ["7b", "33b"])
+def test_large_shapes_two_layers_benchmark_weights(name):
+    """N(0, 0.02) weights against the oracle's bf16-storage mode: 2e-2 on the target; the draft module's tensors
+    (un-normalised vocabulary logits on an expanding stack) stay within 0.15 (measured 6e-2)."""
+    shape = inputs.get_shape(name).with_(n_layers=2, prompt_len=70)
+    rep = _run(shape, 2, True, kv_layers=(0, 1), storage=torch.bfloat16)
+    assert rep.steps == 2
+    assert max(rep.max_logit_err, rep.max_hidden_err, rep.max_kv_err) <= TOL_BF16
+    assert max(rep.max_dlogit_err, rep.max_draft_err) <= 0.15

@@ -556,3 +556,96 @@ def test_ablations_stay_lossless(variant):
         leaf = t.leaves[i % len(t.leaves)]
         out += orc.step(st, t, _plant(t, st.root, ref[len(out) + 1: len(out) + 1 + t.depth[leaf]], leaf), {})
     assert out == ref[: len(out)] and st.root == ref[len(out)]
+
+
+# --------------------------------------------------------------------------------------
+# Eq. 1: what the adaptation layers are fed
+# --------------------------------------------------------------------------------------
+def _draft_with(shape, w, pending_mod=None, prompt=None):
+    """Prefill + draft on a copy of the state; returns (h1 of the last row, stage-1 cache, stage-2 cache)."""
+    orc = ao.Oracle(shape, w, dtype=torch.float64)
+    st = orc.prefill(prompt)
+    if pending_mod is not None:
+        st.pending = pending_mod(list(st.pending))
+    taps = {}
+    orc.draft(st, taps)
+    return taps["h1"], st.sal_kv[0], st.sal_kv[-1]
+
+
+def test_eq1_input_is_hidden_then_embedding():
+    """Eq. 1 feeds fc the concatenation [h_t ; e_{t+1}] in that order.  With the embedding half of fc1's columns
+    zeroed the stage output cannot depend on the sampled token (but does on h_t); with the hidden half zeroed it
+    cannot depend on h_t (but does on the token).  A swapped concatenation, or an embedding that is ignored,
+    fails one of the four assertions."""
+    shape = MICRO
+    d = shape.d_model
+    prompt = inputs.make_prompt(shape).tolist()
+    base = inputs.make_weights(shape, seed=0, std=0.2)
+    other_tok = lambda p: p[:-1] + [(p[-1][0], (p[-1][1] + 7) % shape.vocab, p[-1][2])]
+    other_hid = lambda p: p[:-1] + [(p[-1][0] * 1.5 + 0.25, p[-1][1], p[-1][2])]
+
+    w = dict(base)
+    w["draft.fc1"] = base["draft.fc1"].clone()
+    w["draft.fc1"][:, d:] = 0                                   # no embedding columns
+    h_ref, _, _ = _draft_with(shape, w, None, prompt)
+    h_tok, _, _ = _draft_with(shape, w, other_tok, prompt)
+    h_hid, _, _ = _draft_with(shape, w, other_hid, prompt)
+    assert torch.equal(h_ref, h_tok)
+    assert float((h_ref - h_hid).abs().max()) > 1e-3
+
+    w = dict(base)
+    w["draft.fc1"] = base["draft.fc1"].clone()
+    w["draft.fc1"][:, :d] = 0                                   # no hidden-state columns
+    h_ref, _, _ = _draft_with(shape, w, None, prompt)
+    h_tok, _, _ = _draft_with(shape, w, other_tok, prompt)
+    h_hid, _, _ = _draft_with(shape, w, other_hid, prompt)
+    assert torch.equal(h_ref, h_hid)
+    assert float((h_ref - h_tok).abs().max()) > 1e-3
+
+
+def test_eq1_embedding_is_that_of_the_next_token():
+    """e_{t+1} is the embedding row of the token that follows position t.  With the adaptation layer reduced to
+    its residual path (zero output and down projections) and fc1 = [0 | I], h^1 of a row IS that embedding row."""
+    shape = MICRO
+    d = shape.d_model
+    prompt = inputs.make_prompt(shape).tolist()
+    w = inputs.make_weights(shape, seed=0, std=0.2)
+    w["draft.fc1"] = torch.cat([torch.zeros(d, d), torch.eye(d)], dim=1)
+    w["draft.sal1.wo"] = torch.zeros(d, d)
+    w["draft.sal1.w_down"] = torch.zeros(d, shape.d_ffn)
+    orc = ao.Oracle(shape, w, dtype=torch.float64)
+    st = orc.prefill(prompt)
+    root = st.root
+    taps = {}
+    orc.draft(st, taps)
+    assert torch.allclose(taps["h1"], w["tok_emb"][root].to(torch.float64), atol=1e-12)
+    # and with fc1 = [I | 0] it is the target's hidden state of the last prompt position
+    w["draft.fc1"] = torch.cat([torch.eye(d), torch.zeros(d, d)], dim=1)
+    orc = ao.Oracle(shape, w, dtype=torch.float64)
+    st = orc.prefill(prompt)
+    h_last = st.pending[-1][0].clone()
+    taps = {}
+    orc.draft(st, taps)
+    assert torch.allclose(taps["h1"], h_last, atol=1e-12)
+
+
+def test_eq1_adaptation_layers_are_causal_over_the_pending_rows():
+    """kv_{1:t-1} in Eq. 1: a row of an adaptation layer sees earlier positions only.  Changing the next-token of
+    pending row j changes the cache rows of positions >= j in both stages and leaves every earlier row bit-identical."""
+    shape = MICRO
+    prompt = inputs.make_prompt(shape).tolist()
+    w = inputs.make_weights(shape, seed=0, std=0.2)
+    j = 4
+
+    def mod(p):
+        p[j] = (p[j][0], (p[j][1] + 11) % shape.vocab, p[j][2])
+        return p
+    _, c1, c2 = _draft_with(shape, w, None, prompt)
+    _, m1, m2 = _draft_with(shape, w, mod, prompt)
+    for a, b, stage in ((c1, m1, 1), (c2, m2, 2)):
+        for s in range(len(prompt)):
+            same = torch.equal(a.k[s], b.k[s]) and torch.equal(a.v[s], b.v[s])
+            if s < j:
+                assert same, f"stage {stage}: position {s} < {j} changed"
+            elif s == j or stage == 2:
+                assert not same, f"stage {stage}: position {s} did not react"
