@@ -54,7 +54,10 @@ enum {
   AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
   AMPH_FLAG_NO_GRAPH = 2,       /* launch kernels one by one instead of replaying a CUDA graph */
   AMPH_FLAG_SEPARATE_MERGE = 8,  /* merge the attention KV splits in a kernel of its own (bf16: a cluster does it otherwise) */
-  AMPH_FLAG_SEPARATE_SWIGLU = 16 /* SwiGLU as a kernel of its own (bf16: the gate / up projection applies it otherwise) */
+  AMPH_FLAG_SEPARATE_SWIGLU = 16, /* SwiGLU as a kernel of its own (bf16: the gate / up projection applies it otherwise) */
+  AMPH_FLAG_NO_SAMPLED_TOKEN = 64, /* the "w/o Sampled-Token" ablation (Section 4.5): the adaptation layers are fed the
+                                    * hidden state alone; draft.fc{s} is then [d, d] instead of [d, 2d]            */
+  AMPH_FLAG_MMA_SYNC_ATTENTION = 32 /* bf16 tree attention on the warp-level mma.sync kernel instead of the tcgen05 / TMA one */
 };
 
 #define AMPH_MAX_HEADS_K 8
@@ -128,7 +131,7 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
 /* Registers the weights.  Names (i = layer, s = 1..n_sal, k = 0..K-1, l = 0..aeb_layers-1):
  *   tok_emb [V,d]; layers.{i}.{attn_norm [d], wq, wk, wv, wo [d,d], ffn_norm [d],
  *   w_gate, w_up [F,d], w_down [d,F]}; final_norm [d]; lm_head [V,d];
- *   draft.fc{s} [d,2d] (Eq. 1; input order [hidden ; token embedding]);
+ *   draft.fc{s} [d,2d] (Eq. 1; input order [hidden ; token embedding]; [d,d] with AMPH_FLAG_NO_SAMPLED_TOKEN);
  *   draft.sal{s}.<the nine per-layer names>; draft.mlp.{k}.w [d,d], draft.mlp.{k}.b [d] (Eq. 2);
  *   draft.pe [K,d] (Eq. 4); draft.aeb.{l}.{wq,wk,wv,wo} [d,d] (Eq. 5); draft.lm_head.{k} [V,d] (Eq. 6),
  *   or with lm_rank = r > 0: draft.lm_head.{k}.a [r,d] and draft.lm_head.{k}.b [V,r] (Appendix A.2.4).
@@ -191,6 +194,16 @@ amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, si
  * device-side errors (AMPH_ERR_TIMEOUT). */
 amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending);
 
+/* Teacher forcing (the counterpart of amph_get_state): replaces the decoding state of a prefilled sequence that has no
+ * draft in flight.  ctx_len: committed tokens (the KV caches of the target and of the adaptation layers are NOT touched:
+ * the caller vouches that their first ctx_len, resp. ctx_len - n_pending, slots belong to the sequence); root: the
+ * token chosen for position ctx_len; the n_pending (1..K+1) rows queued for the adaptation layers (Eq. 1) sit at
+ * positions ctx_len - n_pending .. ctx_len - 1: pend_hidden f32 [n_pending][d_model] (host or device) holds the
+ * target's post-final-norm hidden rows h_j, pend_next (HOST, n_pending ids) the token at position j + 1 of each
+ * (the last one is root).  Synchronises the stream. */
+amph_status amph_set_state(amph_ctx* ctx, int32_t ctx_len, int32_t root, int32_t n_pending, const float* pend_hidden,
+                           const int32_t* pend_next);
+
 /* Per-kernel timing of the projections (the weight-streaming kernels that dominate a step).
  * Between amph_profile_begin and amph_profile_end every projection launch is bracketed by CUDA
  * events on the context's stream.  amph_profile_end synchronises the stream and reports, summed over
@@ -224,6 +237,16 @@ amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launc
 amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
                          int32_t out, int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core,
                          float* y_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
+/* Failure-path self-test of the bounded device-side waits (no counterpart in the paper).  Runs the tensor-core
+ * projection of amph_project (bf16, same arguments) with every pipeline wait limited to limit_us microseconds and the
+ * first pipeline barrier of each CTA expecting 1 KB more than its copies deliver, so that this wait can never
+ * complete.  Nothing faults and nothing hangs: each CTA gives up after the limit, lets its own copies land, frees its
+ * tensor memory and returns; y_dev receives zeros.  After the stream has been synchronised the first int32 of ws_dev
+ * reads AMPH_ERR_TIMEOUT.  The device context stays usable. */
+amph_status amph_selftest_wait_timeout(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
+                                       int32_t out, int32_t in, int32_t rows, float* y_dev, void* ws_dev, size_t ws_bytes,
+                                       void* stream, int32_t limit_us);
 
 /* (No counterpart in the paper: a packaging variant of amph_project.)
  * The same projection for callers that cannot allocate device memory at the time of the call: for

@@ -25,6 +25,7 @@ class ModelShape:
     n_sal: int = 2        # staged adaptation layers (Section 3.1)
     aeb_layers: int = 1   # self-attention layers in the Auto-embedding Block
     lm_rank: int = 0      # 0: full drafting vocabulary heads; r > 0: each head is B[V, r] . A[r, d] (Appendix A.2.4)
+    use_sampled_token: bool = True   # False: the "w/o Sampled-Token" ablation of Section 4.5 (fc: d -> d on the hidden state alone)
     topk: Tuple[int, ...] = (10, 10, 10, 10)   # candidates kept per head
     n_nodes: int = 64     # tree nodes including the root
     prompt_len: int = 512

@@ -138,7 +138,7 @@ def weight_specs(shape: ModelShape) -> List[Tuple[str, Tuple[int, ...], str]]:
         specs += _layer_specs(f"layers.{i}.", d, f)
     specs += [("final_norm", (d,), "ones"), ("lm_head", (v, d), "normal")]
     for s in range(1, shape.n_sal + 1):
-        specs.append((f"draft.fc{s}", (d, 2 * d), "normal"))
+        specs.append((f"draft.fc{s}", (d, 2 * d if shape.use_sampled_token else d), "normal"))
         specs += _layer_specs(f"draft.sal{s}.", d, f)
     for k in range(K):
         specs.append((f"draft.mlp.{k}.w", (d, d), "normal"))

@@ -287,8 +287,11 @@ class Oracle:
         feats = [h for (h, _, _) in st.pending]
         for stage in range(1, s.n_sal + 1):
             fc = self.W(f"draft.fc{stage}")
-            X = torch.stack([fc @ self.st(torch.cat([f, self.embed(nxt)]))   # Eq. 1: fc([h ; e_{t+1}])
-                             for (h, nxt, pos), f in zip(st.pending, feats)])
+            if getattr(s, "use_sampled_token", True):
+                X = torch.stack([fc @ self.st(torch.cat([f, self.embed(nxt)]))   # Eq. 1: fc([h ; e_{t+1}])
+                                 for (h, nxt, pos), f in zip(st.pending, feats)])
+            else:            # Section 4.5, "w/o Sampled-Token": the stage sees the hidden state alone, fc is d -> d
+                X = torch.stack([fc @ self.st(f) for f in feats])
             poss = [pos for (_, _, pos) in st.pending]
             vis = [list(range(p + 1)) for p in poss]                  # causal: kv_{1:t-1} and itself
             outs = list(self.decoder_rows(f"draft.sal{stage}.", X, poss, poss, vis,

@@ -18,12 +18,13 @@ AMPH_MAX_NODES = 128
 AMPH_TOPK_STRIDE = 16
 AMPH_DTYPE_F32, AMPH_DTYPE_BF16 = 0, 1
 AMPH_FLAG_NO_TENSOR_CORE, AMPH_FLAG_NO_GRAPH = 1, 2
+AMPH_FLAG_SEPARATE_MERGE, AMPH_FLAG_SEPARATE_SWIGLU, AMPH_FLAG_MMA_SYNC_ATTENTION, AMPH_FLAG_NO_SAMPLED_TOKEN = 8, 16, 32, 64
 STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH_ERR_STATE",
           4: "AMPH_ERR_CAPACITY", 5: "AMPH_ERR_WORKSPACE", 6: "AMPH_ERR_MISSING_WEIGHT",
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
 EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
-           "amph_get_state", "amph_profile_begin", "amph_profile_end", "amph_profile_breakdown", "amph_project", "amph_project_noalloc",
+           "amph_get_state", "amph_set_state", "amph_selftest_wait_timeout", "amph_profile_begin", "amph_profile_end", "amph_profile_breakdown", "amph_project", "amph_project_noalloc",
            "amph_reset", "amph_destroy", "amph_last_error"]
 
 
@@ -83,6 +84,9 @@ def lib() -> C.CDLL:
         L.amph_get_tensor.argtypes = [vp, C.c_char_p, vp, C.c_size_t]
         L.amph_set_tensor.argtypes = [vp, C.c_char_p, vp, C.c_size_t]
         L.amph_get_state.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.amph_set_state.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp, C.POINTER(C.c_int32)]
+        L.amph_selftest_wait_timeout.argtypes = [vp, C.c_int32, C.POINTER(vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                 vp, vp, C.c_size_t, vp, C.c_int32]
         L.amph_profile_begin.argtypes = [vp]
         L.amph_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.amph_profile_breakdown.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -115,7 +119,7 @@ def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0) -> amph_co
     c.lm_rank = getattr(shape, "lm_rank", 0)
     for k in range(shape.K):
         c.topk[k] = shape.topk[k]
-    c.flags = flags
+    c.flags = flags | (0 if getattr(shape, "use_sampled_token", True) else AMPH_FLAG_NO_SAMPLED_TOKEN)
     return c
 
 
@@ -239,6 +243,17 @@ class Amphista:
             self._check(self.L.amph_get_state(self.ctx, C.byref(a), C.byref(b), C.byref(c)), self.ctx)
         return a.value, b.value, c.value
 
+    def set_state(self, ctx_len: int, root: int, pend_hidden: torch.Tensor, pend_next: Sequence[int]) -> None:
+        """amph_set_state: pend_hidden f32 [n_pending, d] (cpu or cuda), pend_next the token after each pending row."""
+        n = len(pend_next)
+        h = pend_hidden.to(torch.float32).contiguous()
+        assert h.shape == (n, self.shape.d_model)
+        ids = (C.c_int32 * n)(*[int(t) for t in pend_next])
+        self._after_torch()
+        with torch.cuda.device(self.device):
+            self._check(self.L.amph_set_state(self.ctx, int(ctx_len), int(root), n, _ptr(h), ids), self.ctx)
+            self.stream.synchronize()                 # h may be a temporary
+
     def profile_begin(self) -> None:
         self._check(self.L.amph_profile_begin(self.ctx), self.ctx)
 
@@ -292,6 +307,24 @@ def project(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, use_tensor_c
     if err:
         raise AmphError(err, "a bounded device-side wait gave up")
     return y
+
+
+def selftest_wait_timeout(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, limit_us: int = 1000):
+    """amph_selftest_wait_timeout: returns (status word read back from the scratch, y)."""
+    L = lib()
+    n_seg = len(ws)
+    out, in_ = ws[0].shape
+    dev = x.device
+    y = torch.full((rows, n_seg * out), float("nan"), dtype=torch.float32, device=dev)
+    scratch = torch.zeros(256 + 16 * 128 * n_seg * out * 4, dtype=torch.uint8, device=dev)
+    arr = (C.c_void_p * n_seg)(*[w.data_ptr() for w in ws])
+    with torch.cuda.device(dev):
+        rc = L.amph_selftest_wait_timeout(_ptr(x), x.shape[0], arr, n_seg, out, in_, rows, _ptr(y), _ptr(scratch),
+                                          scratch.numel(), C.c_void_p(torch.cuda.current_stream(dev).cuda_stream), limit_us)
+        if rc != 0:
+            raise AmphError(rc, L.amph_last_error(None).decode())
+        torch.cuda.synchronize(dev)
+    return int(scratch[:4].view(torch.int32)[0]), y
 
 
 def project_noalloc(x: torch.Tensor, ws: Sequence[torch.Tensor], rows: int, use_tensor_core: bool,

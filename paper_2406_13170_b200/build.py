@@ -7,7 +7,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["amph_api.cu", "kernels.cu", "gemm_tc.cu", "attention_mma.cu", "project_static.cu"]
+SOURCES = ["amph_api.cu", "kernels.cu", "gemm_tc.cu", "attention_mma.cu", "attention_tc.cu", "project_static.cu"]
 LIB = os.path.join(HERE, "libamph.so")
 
 

@@ -77,6 +77,7 @@ struct amph_ctx {
   int ctx_hi;               // host-side upper bound of the committed length
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
+  AttnTc* attn_tc = nullptr; // tcgen05 tree attention (NULL: fp32 caches, disabled or unsupported)
   int sm_count = 148;
   bool last_proj_one_wave = false;   // the last projection ran on the tensor-core kernel with a fully resident grid
   cudaGraphExec_t graph_exec = nullptr;   // captured draft -> verify -> accept schedule of amph_step
@@ -290,7 +291,7 @@ amph_status resolve(amph_ctx* ctx) {
   ctx->layers.resize(c.n_layers);
   for (int i = 0; i < c.n_layers; ++i) resolve_layer(ctx, "layers." + std::to_string(i) + ".", &ctx->layers[i], &ok);
   for (int s = 0; s < c.n_sal; ++s) {
-    ctx->fc[s] = find(ctx, "draft.fc" + std::to_string(s + 1), d, 2 * d, &ok);
+    ctx->fc[s] = find(ctx, "draft.fc" + std::to_string(s + 1), d, (c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN) ? d : 2 * d, &ok);
     resolve_layer(ctx, "draft.sal" + std::to_string(s + 1) + ".", &ctx->sal[s], &ok);
   }
   for (int k = 0; k < c.K; ++k) {
@@ -385,9 +386,20 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   }
   AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
   { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
-  launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
-                        c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr,
-                        (c.flags & AMPH_FLAG_SEPARATE_MERGE) != 0);
+  bool done = false;
+  if (ctx->attn_tc) {
+    const int splits = attn_tc_splits(ctx->attn_tc, ctx_hi, c.n_heads, rows, l.attn_splits);
+    const bool merged = !(c.flags & AMPH_FLAG_SEPARATE_MERGE);
+    done = launch_tree_attention_tc(ctx->attn_tc, ctx->ws + l.q, ctx->Mcap, kv, meta, sc, rows, c.n_heads, c.head_dim, c.max_ctx,
+                                    splits, ctx_hi, st, merged ? ctx->ws + l.att : nullptr, &ctx->at<DevState>(l.state)->err);
+    if (done && !merged)
+      launch_attn_combine(sc, ctx->ws + l.att, ctx->dtype, splits, rows, c.n_heads, c.head_dim, st, ctx->tc != nullptr);
+    if (!done) cudaGetLastError();
+  }
+  if (!done)
+    launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
+                          c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr,
+                          (c.flags & AMPH_FLAG_SEPARATE_MERGE) != 0);
   }
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
@@ -473,10 +485,11 @@ void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, i
   for (int s = 0; s < c.n_sal; ++s) {
     float* hbuf = ctx->at<float>(s == 0 ? l.h1 : l.h2);
     { ProfScope ps(ctx, AMPH_PROF_OTHER);
-    launch_concat(in_feat, ctx->tok_emb, next_tok, c.vocab, ctx->ws + l.cat, ctx->dtype, rows, c.d_model, st);
+    const bool with_tok = !(c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN);             // Section 4.5, "w/o Sampled-Token"
+    launch_concat(in_feat, with_tok ? ctx->tok_emb : nullptr, next_tok, c.vocab, ctx->ws + l.cat, ctx->dtype, rows, c.d_model, st);
     }
     const void* w[1] = {ctx->fc[s]};
-    PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, 2 * c.d_model, rows);
+    PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, ((c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN) ? 1 : 2) * c.d_model, rows);
     { ProfScope ps(ctx, AMPH_PROF_NORM);
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
@@ -595,7 +608,11 @@ amph_status do_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_
   return rc;
 }
 
-int attn_splits_for(const amph_ctx* ctx, int ctx_hi) {
+int attn_splits_for(const amph_ctx* ctx, int ctx_hi, int rows) {
+  if (ctx->attn_tc) {         // split count and ring depth both shape the captured launch
+    const int sp = attn_tc_splits(ctx->attn_tc, ctx_hi, ctx->cfg.n_heads, rows, ctx->lay.attn_splits);
+    return sp * 8 + attn_tc_stages(ctx_hi, sp, ctx->cfg.head_dim);
+  }
   int s = (ctx_hi + 127) / 128;
   if (s > ctx->lay.attn_splits) s = ctx->lay.attn_splits;
   return s < 1 ? 1 : s;
@@ -674,6 +691,9 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   for (int s = 0; s < cfg->n_sal; ++s) { ctx->kv_sal[s].k = p; ctx->kv_sal[s].v = p + half_layer; p += 2 * half_layer; }
   cudaStream_t st = ctx->stream;
   cudaError_t e = cudaMemsetAsync(ctx->ws, 0, l.total, st);
+  // The attention kernels fetch whole key tiles; slots past the live range are masked (probability 0), which only
+  // cancels finite values, so the caches must never hold the NaN patterns of uninitialised memory.
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->kv, 0, need_kv, st);
   std::vector<double> inv(cfg->head_dim / 2);
   for (int i = 0; i < cfg->head_dim / 2; ++i) inv[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.tree, &ctx->tree_host, sizeof(TreeDev), cudaMemcpyHostToDevice, st);
@@ -727,10 +747,13 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
     void* xb[XB_COUNT];
     for (int i = 0; i < XB_COUNT; ++i) xb[i] = xbuf_ptr(ctx, i);
     const int xrows[XB_COUNT] = {ctx->Mcap, ctx->Mcap, ctx->Mcap, ctx->Mcap, 16, 16, 16, 16};
-    const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, 2 * c.d_model, c.d_model, c.d_model, c.d_model,
+    const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, ((c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN) ? 1 : 2) * c.d_model,
+                                 c.d_model, c.d_model, c.d_model,
                                  c.lm_rank > 0 ? c.lm_rank : 8};
     ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
   }
+  if (!ctx->attn_tc && c.kv_dtype == AMPH_DTYPE_BF16 && !(c.flags & AMPH_FLAG_MMA_SYNC_ATTENTION))
+    ctx->attn_tc = attn_tc_create();
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
   const int M = ctx->Mcap;
@@ -808,7 +831,8 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n) {
   if (use_graph) {
     // The kernels read every length from device state; only the attention grids depend on the host's
     // bound of the context length, so the captured schedule is reused until that grid size changes.
-    const int key = attn_splits_for(ctx, ctx->ctx_hi) * 64 + attn_splits_for(ctx, ctx->ctx_hi + ctx->tree_host.n_nodes);
+    const int key = attn_splits_for(ctx, ctx->ctx_hi, ctx->rows_small) * 128 +
+                    attn_splits_for(ctx, ctx->ctx_hi + ctx->tree_host.n_nodes, ctx->Mver);
     if (!ctx->graph_exec || key != ctx->graph_key) {
       if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
       cudaGraph_t graph = nullptr;
@@ -958,9 +982,9 @@ amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launc
   return AMPH_OK;
 }
 
-amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg, int32_t out,
-                         int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core, float* y_dev, void* ws_dev,
-                         size_t ws_bytes, void* stream) {
+static amph_status project_standalone(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg, int32_t out,
+                                      int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core, float* y_dev, void* ws_dev,
+                                      size_t ws_bytes, void* stream, unsigned long long limit_ns, unsigned extra_tx) {
   if (!x_dev || !w || !y_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "NULL pointer");
   if (n_seg < 1 || n_seg > kMaxK || out < 1 || in < 8 || rows < 1 || rows > kMaxRows || x_rows_cap < rows)
     return fail(nullptr, AMPH_ERR_SHAPE, "bad projection shape");
@@ -983,6 +1007,7 @@ amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* cons
     const int xr[1] = {x_rows_cap}, xc[1] = {in};
     TcGemm* g = tc_gemm_create(xb, xr, xc, 1, err);
     if (!g) return fail(nullptr, AMPH_ERR_CUDA, "tensor-map encoder unavailable or not an sm_100 device");
+    if (limit_ns) tc_gemm_set_selftest(g, limit_ns, extra_tx);
     int splits = 0;
     size_t stride = 0;
     const bool ok = tc_gemm_launch(g, 0, w, n_seg, out, in, rows, P, p_floats, &splits, &stride, st);
@@ -999,6 +1024,52 @@ amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* cons
   }
   launch_reduce_partials(pv, y_dev, rows, (int)ld, st);
   return cuda_check(nullptr, cudaGetLastError(), "projection");
+}
+
+amph_status amph_project(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg, int32_t out,
+                         int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core, float* y_dev, void* ws_dev,
+                         size_t ws_bytes, void* stream) {
+  return project_standalone(x_dev, x_rows_cap, w, n_seg, out, in, rows, dtype, use_tensor_core, y_dev, ws_dev, ws_bytes, stream,
+                            0ull, 0u);
+}
+
+amph_status amph_selftest_wait_timeout(const void* x_dev, int32_t x_rows_cap, const void* const* w, int32_t n_seg,
+                                       int32_t out, int32_t in, int32_t rows, float* y_dev, void* ws_dev, size_t ws_bytes,
+                                       void* stream, int32_t limit_us) {
+  if (limit_us < 1 || limit_us > 1000000) return fail(nullptr, AMPH_ERR_INVALID_ARG, "limit_us must be in 1..1000000");
+  return project_standalone(x_dev, x_rows_cap, w, n_seg, out, in, rows, AMPH_DTYPE_BF16, 1, y_dev, ws_dev, ws_bytes, stream,
+                            (unsigned long long)limit_us * 1000ull, 1024u);
+}
+
+amph_status amph_set_state(amph_ctx* ctx, int32_t ctx_len, int32_t root, int32_t n_pending, const float* pend_hidden,
+                           const int32_t* pend_next) {
+  if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (ctx->phase != PH_READY) return fail(ctx, AMPH_ERR_STATE, "amph_set_state needs a prefilled sequence and no draft in flight");
+  const amph_config& c = ctx->cfg;
+  if (!pend_hidden || !pend_next) return fail(ctx, AMPH_ERR_INVALID_ARG, "pend_hidden and pend_next must not be NULL");
+  if (n_pending < 1 || n_pending > c.K + 1 || n_pending > ctx_len)
+    return fail(ctx, AMPH_ERR_INVALID_ARG, "n_pending must be in 1..K+1 and at most ctx_len");
+  if (root < 0 || root >= c.vocab) return fail(ctx, AMPH_ERR_INVALID_ARG, "root %d is outside the vocabulary", root);
+  for (int j = 0; j < n_pending; ++j)
+    if (pend_next[j] < 0 || pend_next[j] >= c.vocab) return fail(ctx, AMPH_ERR_INVALID_ARG, "pend_next[%d] is outside the vocabulary", j);
+  if (ctx_len + ctx->tree_host.n_nodes > c.max_ctx)
+    return fail(ctx, AMPH_ERR_CAPACITY, "ctx_len %d + %d tree nodes exceeds max_ctx %d", ctx_len, ctx->tree_host.n_nodes, c.max_ctx);
+  DevState s;
+  memset(&s, 0, sizeof s);
+  s.C = ctx_len;
+  s.root = root;
+  s.n_pending = n_pending;
+  for (int j = 0; j < n_pending; ++j) s.pend_tok[j] = pend_next[j];
+  s.C_old = ctx_len;
+  s.next_root = root;
+  for (int j = 0; j < 16; ++j) { s.path[j] = -1; s.out_tok[j] = -1; }
+  amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<DevState>(ctx->lay.state), &s, sizeof s, cudaMemcpyHostToDevice, ctx->stream), "set_state");
+  if (rc == AMPH_OK) rc = cuda_check(ctx, cudaStreamSynchronize(ctx->stream), "set_state");       // s lives on this stack frame
+  if (rc == AMPH_OK)
+    rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<float>(ctx->lay.pend_h), pend_hidden, sizeof(float) * (size_t)n_pending * c.d_model,
+                                         cudaMemcpyDefault, ctx->stream), "set_state");
+  if (rc == AMPH_OK) ctx->ctx_hi = ctx_len;
+  return rc;
 }
 
 amph_status amph_profile_breakdown(amph_ctx* ctx, double* ms, int64_t* launches) {
@@ -1021,6 +1092,7 @@ amph_status amph_reset(amph_ctx* ctx) {
 void amph_destroy(amph_ctx* ctx) {
   if (!ctx) return;
   if (ctx->tc) tc_gemm_destroy(ctx->tc);
+  if (ctx->attn_tc) attn_tc_destroy(ctx->attn_tc);
   if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
   for (auto& e : ctx->prof_ev) cudaEventDestroy(e);
   delete ctx;

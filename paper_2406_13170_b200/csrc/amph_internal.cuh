@@ -161,6 +161,19 @@ void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnSc
 bool launch_tree_attention_mma(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
                                int head_dim, int max_ctx, int splits, cudaStream_t st, void* merged_out);
 
+void launch_attn_combine(AttnScratch sc, void* out, int dtype, int splits, int rows, int n_heads, int head_dim,
+                         cudaStream_t st, int early);
+
+// tcgen05 / TMA tree attention (bf16 caches).  An AttnTc holds the tensor maps of the caches it has seen.
+struct AttnTc;
+AttnTc* attn_tc_create();
+void attn_tc_destroy(AttnTc* a);
+int attn_tc_splits(const AttnTc* a, int keys_bound, int n_heads, int rows, int max_splits);
+int attn_tc_stages(int keys_bound, int splits, int head_dim);
+bool launch_tree_attention_tc(AttnTc* a, const void* q, int q_rows_cap, KvView kv, const RowMeta* meta, AttnScratch sc, int rows,
+                              int n_heads, int head_dim, int max_ctx, int splits, int keys_bound, cudaStream_t st,
+                              void* merged_out, int* err_flag);
+
 void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale(),
                    int early = 0);
 

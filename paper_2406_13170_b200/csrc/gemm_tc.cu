@@ -55,6 +55,8 @@ struct TcParams {
   int up_first;             // the tensor map's outer index 0 is the up matrix (it has the lower address)
   RowScale rs;
   int* err_flag;
+  unsigned long long wait_limit_ns;   // a barrier wait gives up after this long
+  uint32_t extra_tx;                   // self-test only: bytes the first stage's barrier expects beyond what is copied
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -83,14 +85,15 @@ __device__ __forceinline__ unsigned long long now_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = now_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try(bar, parity)) return true;
     if ((i & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (now_ns() - t0 > kWaitLimitNs) break;
+      if (now_ns() - t0 > limit_ns) break;
     }
   }
   *abort_flag = 1;
@@ -194,6 +197,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   __shared__ int abort_flag;
 
   pdl_launch_dependents();                          // the consumer kernel may get resident and wait
+  const unsigned long long limit_ns = prm.wait_limit_ns;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
@@ -245,7 +249,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     const int npf = nit < npre + prm.l2_prefetch ? nit : npre + prm.l2_prefetch;
     if (leader) {
       for (int i = 0; i < npre; ++i) {
-        mbar_expect_tx(&full_bar[i], a_bytes + b_bytes);
+        // extra_tx is 0 except in the failure-path self-test, where the first barrier expects bytes that never come
+        mbar_expect_tx(&full_bar[i], a_bytes + b_bytes + (i == 0 ? prm.extra_tx : 0u));
         if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
         else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
       }
@@ -264,7 +269,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     int issued = npre;
     for (int i = npre; i < nit; ++i) {
       const int s = i % stages, round = i / stages;
-      if (!__all_sync(0xffffffffu, mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag, limit_ns))) break;
       if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
@@ -280,7 +285,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       for (int i = first; i < issued; ++i) {
         const int s = i % stages, round = i / stages;
         const unsigned long long t0 = now_ns();
-        while (!mbar_try(&full_bar[s], round & 1) && now_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try(&full_bar[s], round & 1) && now_ns() - t0 < limit_ns) {}
       }
     }
   } else if (warp == 1) {
@@ -290,7 +295,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     bool ok = true;
     for (int i = 0; i < nit; ++i) {
       const int s = i % stages, round = i / stages;
-      ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, &abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(&full_bar[s], round & 1, &abort_flag, limit_ns));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       if (leader) {
@@ -331,7 +336,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       if (et < prm.rows) inv_s[et] = row_scale(prm.rs, et);
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag) : false);
+    const bool ok = __all_sync(0xffffffffu, nkb > 0 ? mbar_wait(&accum_bar, 0, &abort_flag, limit_ns) : false);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if constexpr (SWIGLU) {
       // lanes 0..15 of the warp of quarter q hold features 16 q .. 16 q + 15 of the tile (gate and up alike); the
@@ -425,6 +430,8 @@ struct TcGemm {
   std::map<std::tuple<const void*, int, int, int, int>, CUtensorMap> cache;   // (ptr, rows, cols, box rows, box K blocks)
   int sm_count = 148;
   int max_smem = 0;
+  unsigned long long wait_limit_ns = kWaitLimitNs;
+  uint32_t extra_tx = 0;
   std::map<std::tuple<const void*, const void*, int, int, int>, CUtensorMap> pair_cache;   // (lower, upper matrix, rows, cols, K blocks)
 
   // Two [rows, cols] matrices as one 4-D tensor (column, row, K block, matrix): a box of 64 rows of both.
@@ -540,6 +547,8 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   // 1 stage measured best (0: +0.7 %, 2: +1.2 %, the former 40 MB budget: +3 % on the step).
   prm.l2_prefetch = 1;
   prm.err_flag = g->err_flag;
+  prm.wait_limit_ns = g->wait_limit_ns;
+  prm.extra_tx = g->extra_tx;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   launch_pdl(tc_gemm_kernel<false>, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
@@ -582,10 +591,16 @@ bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_
   prm.up_first = up_first ? 1 : 0;
   prm.rs = rs;
   prm.err_flag = g->err_flag;
+  prm.wait_limit_ns = g->wait_limit_ns;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   return launch_pdl(tc_gemm_kernel<true>, dim3(tiles, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
 }
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }
+
+void tc_gemm_set_selftest(TcGemm* g, unsigned long long wait_limit_ns, unsigned extra_tx) {
+  g->wait_limit_ns = wait_limit_ns;
+  g->extra_tx = extra_tx;
+}
 
 }  // namespace amph

@@ -29,4 +29,8 @@ bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_
 
 void tc_gemm_destroy(TcGemm* g);
 
+// Failure-path self-test: every barrier wait of later launches gives up after wait_limit_ns, and the first stage's
+// barrier of each CTA expects extra_tx bytes more than its copies deliver (so that wait can never complete).
+void tc_gemm_set_selftest(TcGemm* g, unsigned long long wait_limit_ns, unsigned extra_tx);
+
 }  // namespace amph

@@ -461,6 +461,12 @@ static void tree_attention_t(const void* q, KvView kv, const RowMeta* meta, Attn
                                                                               n_heads, DH, 0);
 }
 
+void launch_attn_combine(AttnScratch sc, void* out, int dtype, int splits, int rows, int n_heads, int head_dim,
+                         cudaStream_t st, int early) {
+  AMPH_DISPATCH(dtype, launch_pdl(attn_combine_kernel<T>, dim3(dim3(rows, n_heads)), dim3(head_dim < 128 ? 64 : 128), 0, st, sc.o, sc.ml,
+                                  (T*)out, splits, rows, n_heads, head_dim, early));
+}
+
 void launch_tree_attention(const void* q, KvView kv, const RowMeta* meta, AttnScratch sc, void* out, int dtype,
                            int rows, int n_heads, int head_dim, int max_ctx, int ctx_hi, int max_splits,
                            cudaStream_t st, int early, int separate_merge) {
@@ -514,17 +520,19 @@ void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStr
 // --------------------------------------------------------------------------------------------
 // Eq. 1's concatenation [feature ; embedding of the next token]
 // --------------------------------------------------------------------------------------------
+// emb == NULL: the ablation without the sampled token; the row is the feature alone (pitch d)
 template <typename T>
 __global__ void concat_kernel(const float* __restrict__ feat, const T* __restrict__ emb,
                               const int* __restrict__ next_tok, int vocab, T* __restrict__ cat, int d) {
   pdl_wait();
   pdl_launch_dependents();
   const int r = blockIdx.x;
+  const size_t pitch = emb ? 2 * (size_t)d : (size_t)d;
   int t = next_tok[r];
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
   for (int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4; c < d; c += gridDim.y * blockDim.x * 4) {
-    store4(cat + (size_t)r * 2 * d + c, load4(feat + (size_t)r * d + c));
-    store4(cat + (size_t)r * 2 * d + d + c, load4(emb + (size_t)t * d + c));
+    store4(cat + (size_t)r * pitch + c, load4(feat + (size_t)r * d + c));
+    if (emb) store4(cat + (size_t)r * pitch + d + c, load4(emb + (size_t)t * d + c));
   }
 }
 

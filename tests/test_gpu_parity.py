@@ -88,16 +88,18 @@ def test_long_prompt_many_attention_splits_bf16():
 
 
 @pytest.mark.parametrize("variant", [dict(n_sal=1), dict(aeb_layers=2), dict(n_sal=1, aeb_layers=2), dict(lm_rank=64),
-                                     dict(lm_rank=24), dict(n_sal=0), dict(aeb_layers=0), dict(n_sal=0, aeb_layers=0)],
+                                     dict(lm_rank=24), dict(n_sal=0), dict(aeb_layers=0), dict(n_sal=0, aeb_layers=0),
+                                     dict(use_sampled_token=False)],
                          ids=["one-sal", "alpha-two-aeb-layers", "one-sal-two-aeb-layers", "low-rank-heads-64",
-                              "low-rank-heads-24", "no-sal", "no-aeb", "no-sal-no-aeb"])
+                              "low-rank-heads-24", "no-sal", "no-aeb", "no-sal-no-aeb", "no-sampled-token"])
 @pytest.mark.parametrize("base", ["tiny", "small_bf16"])
 def test_draft_module_variants(base, variant):
     """The draft-module variants the paper evaluates: a single adaptation layer (the "One-Adaptation-Layer"
     ablation of Section 4.5: every head then reads h1), the two-layer Auto-embedding Block ("Amphista-alpha",
     Appendix A.2.3) and vocabulary heads factored into two low-rank matrices (Appendix A.2.4; on bf16, rank 64
     takes the tensor-core projection and rank 24 the plain one); and the ablations of Section 4.5 that remove a
-    module: no adaptation layers (the heads read the target's hidden state) and no Auto-embedding Block."""
+    module: no adaptation layers (the heads read the target's hidden state), no Auto-embedding Block, and no
+    sampled token (fc is d -> d on the hidden state alone)."""
     shape = inputs.get_shape(base).with_(**variant)
     topo = inputs.make_tree(shape.n_nodes, shape.topk)
     model, orc = _setup(shape, topo)

@@ -542,7 +542,33 @@ def test_variant_without_adaptation_layers_or_auto_embedding():
     assert bool(((two.aeb(Hq) - two.aeb(Hp)).abs().amax(dim=1)[1:] > 1e-8).all())   # with the block, rows do interact
 
 
-@pytest.mark.parametrize("variant", [dict(n_sal=0), dict(aeb_layers=0)], ids=["no-sal", "no-aeb"])
+def test_variant_without_sampled_token():
+    """Section 4.5, "w/o Sampled-Token": fc is d -> d on the hidden state alone, so nothing in the draft module depends
+    on the token sampled from h_t; and it equals the full model whose fc has its embedding columns zeroed."""
+    prompt = inputs.make_prompt(MICRO).tolist()
+    d = MICRO.d_model
+    s0 = MICRO.with_(use_sampled_token=False)
+    specs = {n: shp for n, shp, _ in inputs.weight_specs(s0)}
+    assert specs["draft.fc1"] == (d, d) and specs["draft.fc2"] == (d, d)
+    w0 = inputs.make_weights(s0, seed=0, std=0.2)
+    o0 = ao.Oracle(s0, w0, dtype=torch.float64)
+    st = o0.prefill(prompt)
+    t0 = {}
+    _, _, dl0 = o0.draft(st, t0)
+    st2 = o0.prefill(prompt)
+    st2.pending = [(h, (nxt + 5) % MICRO.vocab, p) for (h, nxt, p) in st2.pending]
+    _, _, dl2 = o0.draft(st2, {})
+    assert torch.equal(dl0, dl2)
+    wf = dict(w0)                                   # the full form with zero embedding columns computes the same thing
+    for sname in ("draft.fc1", "draft.fc2"):
+        wf[sname] = torch.cat([w0[sname], torch.zeros(d, d)], dim=1)
+    of = ao.Oracle(MICRO, wf, dtype=torch.float64)
+    _, _, dlf = of.draft(of.prefill(prompt), {})
+    assert torch.allclose(dl0, dlf, atol=1e-12)
+
+
+@pytest.mark.parametrize("variant", [dict(n_sal=0), dict(aeb_layers=0), dict(use_sampled_token=False)],
+                         ids=["no-sal", "no-aeb", "no-sampled-token"])
 def test_ablations_stay_lossless(variant):
     shape = MICRO.with_(**variant)
     orc = ao.Oracle(shape, inputs.make_weights(shape, seed=0, std=0.2), dtype=torch.float64)
