@@ -230,7 +230,8 @@ amph_status amph_profile_end(amph_ctx* ctx, double* proj_ms, int64_t* proj_launc
  * ([x_rows_cap, in] row-major, device, same dtype as the weights; only the first `rows` are used).
  * w: HOST array of n_seg device pointers.  y: device fp32 [rows, n_seg*out].
  * use_tensor_core != 0 selects the tcgen05 kernel (bf16 only; out % 128 == 0, in % 64 == 0,
- * rows <= 128, x_rows_cap >= rows rounded up to 16) and fails with AMPH_ERR_SHAPE if the shape is
+ * rows <= 512, x_rows_cap >= rows rounded up to 16, or to 128 beyond 128 rows: then every weight tile is streamed once
+ * and multiplied with up to four 128-row blocks) and fails with AMPH_ERR_SHAPE if the shape is
  * not covered; 0 selects the plain CUDA-core kernel.  ws_dev: device scratch of ws_bytes >=
  * 256 + 16 * 128 * n_seg * out * 4 bytes, 256-byte aligned; its first int32 is zeroed by the call and is set to
  * AMPH_ERR_TIMEOUT if a bounded device-side wait gave up.  Stream-ordered; no context needed. */

@@ -986,7 +986,7 @@ static amph_status project_standalone(const void* x_dev, int32_t x_rows_cap, con
                                       int32_t in, int32_t rows, int32_t dtype, int32_t use_tensor_core, float* y_dev, void* ws_dev,
                                       size_t ws_bytes, void* stream, unsigned long long limit_ns, unsigned extra_tx) {
   if (!x_dev || !w || !y_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "NULL pointer");
-  if (n_seg < 1 || n_seg > kMaxK || out < 1 || in < 8 || rows < 1 || rows > kMaxRows || x_rows_cap < rows)
+  if (n_seg < 1 || n_seg > kMaxK || out < 1 || in < 8 || rows < 1 || rows > 4 * kMaxRows || x_rows_cap < rows)
     return fail(nullptr, AMPH_ERR_SHAPE, "bad projection shape");
   if (dtype != AMPH_DTYPE_F32 && dtype != AMPH_DTYPE_BF16) return fail(nullptr, AMPH_ERR_SHAPE, "unknown dtype");
   if (in % (dtype == AMPH_DTYPE_F32 ? 4 : 8)) return fail(nullptr, AMPH_ERR_SHAPE, "in must be a multiple of 16 bytes");

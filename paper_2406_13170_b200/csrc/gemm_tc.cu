@@ -43,7 +43,8 @@ struct TcParams {
   int tiles_per_seg;        // out / 128
   int kblocks;              // in / 64
   int splits;
-  int nt;                   // activation rows in the MMA (multiple of 16)
+  int nt;                   // activation rows of one MMA (multiple of 16, at most 128)
+  int nblk;                 // row blocks of nt rows that share each weight tile (1..4; more than 1 only with nt = 128)
   int rows;                 // live rows (only these are stored)
   int stages;
   int l2_prefetch;          // weight tiles (beyond the ring) each CTA pulls into L2 before it waits
@@ -213,11 +214,14 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int nt = prm.nt, stages = prm.stages;
   const uint32_t a_tile = kTileM * kTileK * 2, b_tile = (uint32_t)nt * kTileK * 2;     // one K block of each operand
   const uint32_t a_bytes = ks * a_tile, b_bytes = ks * b_tile;
-  const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+  const int nblk = SWIGLU ? 1 : prm.nblk;              // row blocks: each gets its own activation tile and accumulator
+  const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
+  const uint32_t stage_bytes = a_bytes + (uint32_t)nblk * b_slot;
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint32_t ntc = 32;
   while ((int)ntc < nt) ntc <<= 1;
-  const uint32_t tmem_cols = SWIGLU ? 2 * ntc : ntc;
+  uint32_t tmem_cols = SWIGLU ? 2 * ntc : ntc * (uint32_t)nblk;
+  if (tmem_cols == 384) tmem_cols = 512;             // allocations are powers of two
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -250,7 +254,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     if (leader) {
       for (int i = 0; i < npre; ++i) {
         // extra_tx is 0 except in the failure-path self-test, where the first barrier expects bytes that never come
-        mbar_expect_tx(&full_bar[i], a_bytes + b_bytes + (i == 0 ? prm.extra_tx : 0u));
+        mbar_expect_tx(&full_bar[i], a_bytes + (uint32_t)nblk * b_bytes + (i == 0 ? prm.extra_tx : 0u));
         if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
         else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
       }
@@ -264,7 +268,8 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     pdl_wait();
     if (leader)
       for (int i = 0; i < npre; ++i)
-        tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[i]);
+        for (int z = 0; z < nblk; ++z)
+          tma_load_3d(smem + (size_t)i * stage_bytes + a_bytes + (size_t)z * b_slot, &maps.x, z * nt, kb_lo + i * ks, &full_bar[i]);
     __syncwarp();
     int issued = npre;
     for (int i = npre; i < nit; ++i) {
@@ -272,10 +277,10 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
       if (!__all_sync(0xffffffffu, mbar_wait(&empty_bar[s], (round & 1) ^ 1, &abort_flag, limit_ns))) break;
       if (leader) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
-        mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+        mbar_expect_tx(&full_bar[s], a_bytes + (uint32_t)nblk * b_bytes);
         if (SWIGLU) tma_load_4d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
         else tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
-        tma_load_3d(a + a_bytes, &maps.x, 0, kb_lo + i * ks, &full_bar[s]);
+        for (int z = 0; z < nblk; ++z) tma_load_3d(a + a_bytes + (size_t)z * b_slot, &maps.x, z * nt, kb_lo + i * ks, &full_bar[s]);
       }
       __syncwarp();
       issued = i + 1;
@@ -316,9 +321,12 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
             }
           } else {
             const uint64_t adesc = umma_desc(a_addr + (uint32_t)kk * a_tile);
+            for (int z = 0; z < nblk; ++z) {             // the weight tile is read from shared memory once per row block
+              const uint64_t bz = umma_desc(a_addr + a_bytes + (uint32_t)z * b_slot + (uint32_t)kk * b_tile);
 #pragma unroll
-            for (int k = 0; k < kTileK / kUmmaK; ++k)    // +32 bytes (2 x 16 B) per K step inside the swizzle row
-              umma_f16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+              for (int k = 0; k < kTileK / kUmmaK; ++k)    // +32 bytes (2 x 16 B) per K step inside the swizzle row
+                umma_f16(tmem_d + (uint32_t)z * ntc, adesc + (uint64_t)(2 * k), bz + (uint64_t)(2 * k), idesc, (i | kk | k) ? 1u : 0u);
+            }
           }
         }
         umma_commit(&empty_bar[s]);                    // frees the stage once these MMAs have read it
@@ -384,25 +392,28 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     } else {
     const int feat = seg * prm.tiles_per_seg * kTileM + row0 + quarter * 32 + lane;
     float* out = prm.P + (size_t)split * prm.split_stride + feat;
-    for (int c0 = 0; c0 < nt; c0 += 16) {
-      if (c0 >= prm.rows) break;
-      uint32_t v[16];
-      if (ok) {
-        const uint32_t taddr = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(taddr)
-            : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      } else {
+    for (int z = 0; z < nblk; ++z) {
+      const int rbase = z * nt;
+      for (int c0 = 0; c0 < nt; c0 += 16) {
+        if (rbase + c0 >= prm.rows) break;
+        uint32_t v[16];
+        if (ok) {
+          const uint32_t taddr = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)z * ntc + (uint32_t)c0;
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+              : "r"(taddr)
+              : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = 0u;          // empty K-range or aborted: contribute zeros
+          for (int j = 0; j < 16; ++j) v[j] = 0u;          // empty K-range or aborted: contribute zeros
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (rbase + c0 + j < prm.rows) out[(size_t)(rbase + c0 + j) * prm.ld] = __uint_as_float(v[j]);
       }
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (c0 + j < prm.rows) out[(size_t)(c0 + j) * prm.ld] = __uint_as_float(v[j]);
     }
     }
   }
@@ -501,21 +512,26 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   if (!g || xb < 0 || xb >= g->n_x) return false;
   if (out % kTileM || in % kTileK || n_seg < 1 || n_seg > kMaxSeg || rows < 1) return false;
   if (g->xcols[xb] != in) return false;
-  const int nt = rows <= 16 ? 16 : (rows + 15) / 16 * 16;
-  if (nt > 128 || nt > g->xrows[xb]) return false;
+  // up to 128 rows: one MMA of N = rows rounded up to 16; more: 2..4 row blocks of 128 rows that share every weight tile
+  // (the tile is streamed from HBM once and multiplied with each block: batched verification, dense prefill)
+  const int nt_all = rows <= 16 ? 16 : (rows <= 128 ? (rows + 15) / 16 * 16 : (rows + 127) / 128 * 128);
+  const int nblk = nt_all <= 128 ? 1 : nt_all / 128;
+  const int nt = nblk == 1 ? nt_all : 128;
+  if (nblk > 4 || nt_all > g->xrows[xb]) return false;
   const int tiles = n_seg * (out / kTileM), kblocks = in / kTileK;
   const size_t ld = (size_t)n_seg * out;
   // K-splits: nearly two CTAs per SM (7/8 of the slots measured best: one split fewer costs no bandwidth and
-  // saves partial sums), keep at least four 64-wide K blocks per CTA
-  int splits = (2 * g->sm_count * 7 / 8) / tiles;
+  // saves partial sums), keep at least four 64-wide K blocks per CTA.  With several row blocks a CTA needs most of an
+  // SM's shared and tensor memory: one CTA per SM.
+  int splits = ((nblk == 1 ? 2 : 1) * g->sm_count * 7 / 8) / tiles;
   if (splits > kblocks / 4) splits = kblocks / 4;
   // many activation rows: a two-block stage would leave room for one CTA per SM only, so stage single blocks
   const int ks = nt <= 64 ? kStageKb : 1;
   if (splits > (kblocks + ks - 1) / ks) splits = (kblocks + ks - 1) / ks;
   if (splits > 16) splits = 16;
-  while (splits > 1 && (size_t)splits * nt * ld > p_floats) --splits;
+  while (splits > 1 && (size_t)splits * nt_all * ld > p_floats) --splits;
   if (splits < 1) splits = 1;
-  if ((size_t)nt * ld > p_floats) return false;
+  if ((size_t)nt_all * ld > p_floats) return false;
   TmapPack pack;
   memset(&pack, 0, sizeof pack);
   for (int s = 0; s < n_seg; ++s) {
@@ -527,13 +543,14 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt, ks);
   if (!mx) return false;
   pack.x = *mx;
-  const uint32_t stage_bytes = ks * kTileM * kTileK * 2 + ((ks * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
-  int stages = (int)((110 * 1024) / stage_bytes);          // <= ~110 KB per CTA: two CTAs per SM
+  const uint32_t stage_bytes = ks * kTileM * kTileK * 2 + (uint32_t)nblk * ((ks * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  int stages = (int)(((nblk == 1 ? 110 : 200) * 1024) / stage_bytes);   // <= ~110 KB per CTA: two CTAs per SM (one with row blocks)
   if (stages > 8) stages = 8;
   if (stages < 2) stages = 2;
   TcParams prm;
   prm.P = P;
-  prm.split_stride = (size_t)nt * ld;
+  prm.nblk = nblk;
+  prm.split_stride = (size_t)nt_all * ld;
   prm.ld = (int)ld;
   prm.tiles_per_seg = out / kTileM;
   prm.kblocks = kblocks;

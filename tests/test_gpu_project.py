@@ -20,6 +20,10 @@ SHAPES = [
     (1, 4096, 4096, 128, 128),    # widest row block
     (1, 4096, 4096, 100, 112),    # ragged rows, cap not a power of two
     (4, 32000, 4096, 4, 16),      # the four drafting vocabulary heads
+    (3, 512, 512, 256, 256),      # two 128-row blocks per weight tile (batched verification)
+    (1, 4096, 4096, 300, 384),    # three blocks, ragged last block
+    (3, 4096, 4096, 512, 512),    # four blocks: a dense prefill pass of 512 rows, 7B q / k / v
+    (2, 1408, 512, 200, 256),
 ]
 
 
