@@ -57,11 +57,13 @@ enum {
   AMPH_FLAG_SEPARATE_SWIGLU = 16, /* SwiGLU as a kernel of its own (bf16: the gate / up projection applies it otherwise) */
   AMPH_FLAG_NO_SAMPLED_TOKEN = 64, /* the "w/o Sampled-Token" ablation (Section 4.5): the adaptation layers are fed the
                                     * hidden state alone; draft.fc{s} is then [d, d] instead of [d, 2d]            */
+  AMPH_FLAG_CHUNKED_PREFILL = 128, /* prefill one chunk of 128 prompt tokens per weight pass instead of four */
   AMPH_FLAG_MMA_SYNC_ATTENTION = 32 /* bf16 tree attention on the warp-level mma.sync kernel instead of the tcgen05 / TMA one */
 };
 
 #define AMPH_MAX_HEADS_K 8
 #define AMPH_MAX_NODES 128
+#define AMPH_MAX_BATCH 8
 #define AMPH_TOPK_STRIDE 16
 
 typedef struct amph_ctx amph_ctx;
@@ -79,7 +81,9 @@ typedef struct {
   int32_t weight_dtype;   /* AMPH_DTYPE_*: storage type of every weight tensor             */
   int32_t kv_dtype;       /* AMPH_DTYPE_*: storage type of all KV caches (must equal weight_dtype) */
   int32_t max_ctx;        /* KV capacity in slots (committed tokens + tree nodes)           */
-  int32_t max_batch;      /* must be 1                                                      */
+  int32_t max_batch;      /* sequences decoded side by side (Section 4.4), 1..AMPH_MAX_BATCH; max_batch * tree nodes
+                           * (rounded up to 16) must not exceed 512.  Every sequence has its own KV caches, length
+                           * and pending rows; one pass streams the weights once for all of them                 */
   int32_t K;              /* drafting heads, 1..AMPH_MAX_HEADS_K (the paper uses 4)         */
   int32_t n_sal;          /* staged adaptation layers: 2 (the paper's design), 1, or 0 (the  *
                            * heads then read the target's hidden state; Section 4.5)         */
@@ -146,6 +150,17 @@ amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t
  * stream before returning.  Resets any previous sequence. */
 amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, int32_t* out_root);
 
+/* The same for sequence seq (0 .. max_batch - 1) of a context created with max_batch > 1 (Section 4.4: several
+ * sequences of different lengths decoded side by side).  Every sequence must be prefilled before the first
+ * amph_draft / amph_step; a sequence may be prefilled again later (between steps) to start a new text in its slot.
+ * With max_batch = B the per-step calls take and return arrays with a leading sequence dimension:
+ *   amph_draft        out_topk_ids / out_topk_vals [B][K][AMPH_TOPK_STRIDE]
+ *   amph_verify_tree  tree_tokens / out_argmax [B][n_nodes]
+ *   amph_accept       out_tokens / out_path [B][K+1], out_n / out_next_root [B]
+ *   amph_step         out_tokens [B][K+1], out_n [B]
+ * Sequences advance independently (own length, own accepted count); one pass streams the weights once for all. */
+amph_status amph_prefill_seq(amph_ctx* ctx, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* out_root);
+
 /* Draft module (Section 3): adaptation layers over the pending rows (Eq. 1), K head MLPs on
  * the last row (Eq. 2), + PE (Eq. 3-4), bi-directional self-attention across the K rows (Eq. 5),
  * K vocabulary projections and top-k (Eq. 6), then tree tokens (Appendix A.1).
@@ -174,9 +189,11 @@ amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int3
  * out_tokens [K+1], out_n [1]: host or device int32, may be NULL. */
 amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n);
 
-/* Debug taps (stream-ordered copy into dst, host or device).  Names and element types:
+/* Debug taps (stream-ordered copy into dst, host or device).  A name may carry "#b" to select sequence b (default 0).
+ * Names and element types:
  *   "hidden" f32 [rows,d] post-final-norm rows of the last target pass and "logits" f32 [rows,V] (rows =
- *   n_nodes after amph_verify_tree; after amph_prefill the rows of its last chunk of AMPH_MAX_NODES prompt tokens);
+ *   n_nodes after amph_verify_tree; after amph_prefill the rows of its last pass: a pass carries 4 * AMPH_MAX_NODES
+ *   prompt tokens, so prompt token j is row j mod 512; AMPH_MAX_NODES with AMPH_FLAG_CHUNKED_PREFILL);
  *   "d_logits" f32 [K,V]; "hp" f32 [K,d] (Eq. 4); "attn_o" f32 [K,d] (Eq. 5);
  *   "sal_h" f32 [2,d] (Eq. 1: h^1_t, h^2_t of the last row); "tree_tokens", "argmax" i32 [n_nodes];
  *   "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v": f32 [rows, d] for cache slots 0..rows-1,
@@ -186,15 +203,17 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
 
 /* Test hook: overwrites "tree_tokens" or "argmax" (i32 [n_nodes], host or device source) with a
  * stream-ordered copy, e.g. to run amph_accept on a chosen verification outcome.  Allowed after
- * amph_verify_tree only.  "root" (i32 [1]) replaces the root token; allowed right after amph_prefill only. */
+ * amph_verify_tree only.  "root" (i32 [1]) replaces the root token; allowed right after amph_prefill only.
+ * "#b" selects the sequence as for amph_get_tensor. */
 amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes);
 
 /* Synchronises the stream and reports the committed length, the current root token and the
  * number of rows pending for the adaptation layers.  Any pointer may be NULL.  Also surfaces
- * device-side errors (AMPH_ERR_TIMEOUT). */
+ * device-side errors (AMPH_ERR_TIMEOUT).  amph_get_state reads sequence 0, amph_get_state_seq sequence seq. */
 amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending);
+amph_status amph_get_state_seq(amph_ctx* ctx, int32_t seq, int32_t* ctx_len, int32_t* root, int32_t* n_pending);
 
-/* Teacher forcing (the counterpart of amph_get_state): replaces the decoding state of a prefilled sequence that has no
+/* Teacher forcing (the counterpart of amph_get_state; sequence 0): replaces the decoding state of a prefilled sequence that has no
  * draft in flight.  ctx_len: committed tokens (the KV caches of the target and of the adaptation layers are NOT touched:
  * the caller vouches that their first ctx_len, resp. ctx_len - n_pending, slots belong to the sequence); root: the
  * token chosen for position ctx_len; the n_pending (1..K+1) rows queued for the adaptation layers (Eq. 1) sit at

@@ -22,7 +22,7 @@ AMPH_FLAG_SEPARATE_MERGE, AMPH_FLAG_SEPARATE_SWIGLU, AMPH_FLAG_MMA_SYNC_ATTENTIO
 STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH_ERR_STATE",
           4: "AMPH_ERR_CAPACITY", 5: "AMPH_ERR_WORKSPACE", 6: "AMPH_ERR_MISSING_WEIGHT",
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}
-EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_draft",
+EXPORTS = ["amph_workspace_bytes", "amph_init", "amph_load_weights", "amph_prefill", "amph_prefill_seq", "amph_get_state_seq", "amph_draft",
            "amph_verify_tree", "amph_accept", "amph_step", "amph_get_tensor", "amph_set_tensor",
            "amph_get_state", "amph_set_state", "amph_selftest_wait_timeout", "amph_profile_begin", "amph_profile_end", "amph_profile_breakdown", "amph_project", "amph_project_noalloc",
            "amph_reset", "amph_destroy", "amph_last_error"]
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
                                 C.c_size_t, vp, C.POINTER(vp)]
         L.amph_load_weights.argtypes = [vp, C.POINTER(amph_tensor), C.c_int32]
         L.amph_prefill.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32)]
+        L.amph_prefill_seq.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32)]
+        L.amph_get_state_seq.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.amph_draft.argtypes = [vp, i32p, f32p]
         L.amph_verify_tree.argtypes = [vp, i32p, i32p]
         L.amph_accept.argtypes = [vp, i32p, i32p, i32p, i32p]
@@ -106,7 +108,7 @@ def lib() -> C.CDLL:
     return _lib
 
 
-def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0) -> amph_config:
+def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0, max_batch: int = 1) -> amph_config:
     """amph_config from an object with the fields of inputs.configs.ModelShape."""
     c = amph_config()
     c.n_layers, c.d_model, c.n_heads, c.head_dim = shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim
@@ -114,7 +116,7 @@ def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0) -> amph_co
     dt = AMPH_DTYPE_F32 if shape.dtype == "fp32" else AMPH_DTYPE_BF16
     c.weight_dtype = c.kv_dtype = dt
     c.max_ctx = int(max_ctx or shape.ctx_capacity)
-    c.max_batch = 1
+    c.max_batch = int(max_batch)
     c.K, c.n_sal, c.aeb_layers = shape.K, shape.n_sal, shape.aeb_layers
     c.lm_rank = getattr(shape, "lm_rank", 0)
     for k in range(shape.K):
@@ -146,11 +148,13 @@ class Amphista:
     """One decoding context.  Owns the device regions (torch tensors) the C library borrows."""
 
     def __init__(self, shape, topo, weights: Dict[str, torch.Tensor], device="cuda:0",
-                 max_ctx: Optional[int] = None, flags: int = 0, stream: Optional[torch.cuda.Stream] = None):
+                 max_ctx: Optional[int] = None, flags: int = 0, stream: Optional[torch.cuda.Stream] = None,
+                 max_batch: int = 1):
         self.L = lib()
         self.shape, self.topo = shape, topo
         self.device = torch.device(device)
-        self.cfg = make_config(shape, max_ctx, flags)
+        self.B = int(max_batch)
+        self.cfg = make_config(shape, max_ctx, flags, max_batch)
         self.tree = make_tree(topo)
         kvb, wsb = C.c_size_t(), C.c_size_t()
         self._check(self.L.amph_workspace_bytes(C.byref(self.cfg), C.byref(self.tree.c), C.byref(kvb), C.byref(wsb)), None)
@@ -167,8 +171,8 @@ class Amphista:
         self.weights = weights            # keeps the tensors alive
         self.load_weights(weights)
         N, K = topo.n_nodes, shape.K
-        self.out_tokens = torch.empty(K + 1, dtype=torch.int32, device=self.device)
-        self.out_n = torch.empty(1, dtype=torch.int32, device=self.device)
+        self.out_tokens = torch.empty(self.B, K + 1, dtype=torch.int32, device=self.device)
+        self.out_n = torch.empty(self.B, dtype=torch.int32, device=self.device)
 
     def _after_torch(self) -> None:
         """Orders the library's stream after work torch has queued on its current stream (inputs)."""
@@ -197,12 +201,12 @@ class Amphista:
         self._after_torch()
         self._check(self.L.amph_load_weights(self.ctx, arr, len(weights)), self.ctx)
 
-    def prefill(self, prompt: Sequence[int]) -> int:
+    def prefill(self, prompt: Sequence[int], seq: int = 0) -> int:
         n = len(prompt)
         ids = (C.c_int32 * n)(*[int(t) for t in prompt])
         root = C.c_int32()
         with torch.cuda.device(self.device):
-            self._check(self.L.amph_prefill(self.ctx, ids, n, C.byref(root)), self.ctx)
+            self._check(self.L.amph_prefill_seq(self.ctx, int(seq), ids, n, C.byref(root)), self.ctx)
         return root.value
 
     def draft(self, out_ids: Optional[torch.Tensor] = None, out_vals: Optional[torch.Tensor] = None) -> None:
@@ -237,10 +241,10 @@ class Amphista:
             self._check(self.L.amph_set_tensor(self.ctx, name.encode(), _ptr(src), src.numel() * src.element_size()),
                         self.ctx)
 
-    def get_state(self):
+    def get_state(self, seq: int = 0):
         a, b, c = C.c_int32(), C.c_int32(), C.c_int32()
         with torch.cuda.device(self.device):
-            self._check(self.L.amph_get_state(self.ctx, C.byref(a), C.byref(b), C.byref(c)), self.ctx)
+            self._check(self.L.amph_get_state_seq(self.ctx, int(seq), C.byref(a), C.byref(b), C.byref(c)), self.ctx)
         return a.value, b.value, c.value
 
     def set_state(self, ctx_len: int, root: int, pend_hidden: torch.Tensor, pend_next: Sequence[int]) -> None:

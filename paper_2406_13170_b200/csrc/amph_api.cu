@@ -28,7 +28,15 @@ struct TensorRec {
   int64_t shape[2];
 };
 
-// Offsets of every buffer inside the caller's workspace region.
+constexpr int kPrefillRows = kMaxRows;           // rows of one prefill chunk (one row group)
+constexpr int kMaxSeq = AMPH_MAX_BATCH;       // sequences of a context = row groups of a batched pass
+constexpr int kPrefillGroups = 4;               // row groups (chunks of 128 prompt tokens) one prefill pass carries
+constexpr int kSmallRows = 16;                  // rows one sequence contributes to the draft module's passes
+
+// Offsets of every buffer inside the caller's workspace region.  A forward pass carries G row groups of equal
+// height: the sequences of a batch (each with its own caches, row table and state) or consecutive chunks of one
+// prompt.  Buffers marked "per group" hold kMaxSeq copies `*_stride` bytes apart; row buffers hold all groups'
+// rows back to back (group g starts at row g * rows-per-group of that pass).
 struct Layout {
   size_t total = 0;
   size_t take(size_t bytes) {
@@ -36,11 +44,19 @@ struct Layout {
     total += (bytes + 255) / 256 * 256;
     return off;
   }
-  size_t state, tree, meta_v, meta_s, kv_tab, inv_freq, rope_v, rope_s;
-  size_t tok, amax, override_tok, next_tok, topk_ids, topk_vals, topk_cand, amax_cand;
-  size_t x, hidden, h1, h2, pend_h, last, hp, attn_o;
-  size_t xn, q, att, act, cat, last_act, ao_act, aeb_act, lr_act;
-  size_t partial, att_o, att_ml, logits, d_logits, ss_a, ss_b;
+  size_t per_group(size_t bytes, size_t* stride) {
+    *stride = (bytes + 255) / 256 * 256;
+    return take(*stride * kMaxSeq);
+  }
+  // per group
+  size_t state, meta_v, meta_s, kv_tab, rope_v, rope_s, topk_ids, topk_vals, topk_cand, last, d_logits, att_o, att_ml;
+  size_t state_s, meta_s_, kv_tab_s, rope_s_, topk_ids_s, topk_vals_s, topk_cand_s, last_s, d_logits_s, att_o_s, att_ml_s;
+  // shared
+  size_t tree, inv_freq;
+  size_t tok, amax, override_tok, next_tok, amax_cand;                  // [Rcap] ints / candidates
+  size_t x, hidden, h1, h2, pend_h, hp, attn_o;                           // fp32 rows
+  size_t xn, q, att, act, cat, last_act, ao_act, aeb_act, lr_act;        // storage-type rows
+  size_t partial, logits, ss_a, ss_b;
   size_t partial_floats;
   int attn_splits;
 };
@@ -55,14 +71,17 @@ struct amph_ctx {
   cudaStream_t stream;
   int dtype;
   size_t esz;
-  int Mcap;                 // row capacity of the activation buffers = rows of a prefill chunk
-  int Mver;                 // rows carried by a verification pass (tree nodes rounded up to 16)
-  int rows_small;           // rows carried by the draft module's passes
+  int B;                    // sequences of this context (cfg.max_batch)
+  int Mcap;                 // rows of one group at most = rows of a prefill chunk
+  int Rcap;                 // rows of one pass at most (all groups)
+  int Mver;                 // rows one sequence carries in a verification pass (tree nodes rounded up to 16)
+  int rows_small;           // rows one sequence carries in the draft module's passes
+  int small_cap;            // row capacity of the draft module's small activation buffers
   Layout lay;
   char* ws;
   char* kv;
-  std::vector<KvView> kv_target;
-  KvView kv_sal[2];
+  std::vector<KvView> kv_target[kMaxSeq];
+  KvView kv_sal[kMaxSeq][2];
   std::unordered_map<std::string, TensorRec> tensors;
   bool resolved;
   const void *tok_emb, *final_norm, *lm_head, *fc[2], *pe;
@@ -74,14 +93,15 @@ struct amph_ctx {
   const void* draft_lm[kMaxK];      // [V, d] heads, or with lm_rank > 0 the [V, r] factors
   const void* draft_lm_a[kMaxK];    // [r, d] factors (lm_rank > 0)
   Phase phase;
-  int ctx_hi;               // host-side upper bound of the committed length
+  bool prefilled[kMaxSeq] = {false};
+  int ctx_hi[kMaxSeq] = {0};   // host-side upper bound of each sequence's committed length
   std::string err;
   TcGemm* tc;               // tensor-core projection plans (NULL when disabled / unsupported)
   AttnTc* attn_tc = nullptr; // tcgen05 tree attention (NULL: fp32 caches, disabled or unsupported)
   int sm_count = 148;
   bool last_proj_one_wave = false;   // the last projection ran on the tensor-core kernel with a fully resident grid
   cudaGraphExec_t graph_exec = nullptr;   // captured draft -> verify -> accept schedule of amph_step
-  int graph_key = -1;       // attention split counts the captured grids were sized for
+  long long graph_key = -1; // attention split counts the captured grids were sized for
   bool graph_off = false;   // capture is not possible (legacy stream, flag) or failed once
   bool prof_on = false;     // bracket projection launches with events (amph_profile_begin / end)
   std::vector<cudaEvent_t> prof_ev;
@@ -92,6 +112,11 @@ struct amph_ctx {
   int64_t prof_cat_n[AMPH_PROF_CATEGORIES] = {0};
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  template <typename T> T* grp(size_t off, size_t stride, int g) const { return reinterpret_cast<T*>(ws + off + stride * g); }
+  DevState* state(int b) const { return grp<DevState>(lay.state, lay.state_s, b); }
+  RowMeta* meta_v(int g) const { return grp<RowMeta>(lay.meta_v, lay.meta_s_, g); }
+  RowMeta* meta_s(int g) const { return grp<RowMeta>(lay.meta_s, lay.meta_s_, g); }
+  int max_ctx_hi() const { int m = 0; for (int b = 0; b < B; ++b) m = ctx_hi[b] > m ? ctx_hi[b] : m; return m; }
 };
 
 namespace {
@@ -146,7 +171,7 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   if (c->weight_dtype != AMPH_DTYPE_F32 && c->weight_dtype != AMPH_DTYPE_BF16)
     return fail(nullptr, AMPH_ERR_SHAPE, "unknown weight_dtype %d", c->weight_dtype);
   if (c->kv_dtype != c->weight_dtype) return fail(nullptr, AMPH_ERR_SHAPE, "kv_dtype must equal weight_dtype");
-  if (c->max_batch != 1) return fail(nullptr, AMPH_ERR_SHAPE, "max_batch must be 1");
+  if (c->max_batch < 1 || c->max_batch > kMaxSeq) return fail(nullptr, AMPH_ERR_SHAPE, "max_batch must be in 1..%d", kMaxSeq);
   if (c->K < 1 || c->K > kMaxK) return fail(nullptr, AMPH_ERR_SHAPE, "K must be in 1..%d", kMaxK);
   if (c->n_sal < 0 || c->n_sal > 2) return fail(nullptr, AMPH_ERR_SHAPE, "n_sal must be 0, 1 or 2");
   if (c->aeb_layers < 0 || c->aeb_layers > 2) return fail(nullptr, AMPH_ERR_SHAPE, "aeb_layers must be 0, 1 or 2");
@@ -157,6 +182,8 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 1.f)) return fail(nullptr, AMPH_ERR_SHAPE, "bad rms_eps / rope_theta");
   if (t->n_nodes < 1 || t->n_nodes > kMaxRows) return fail(nullptr, AMPH_ERR_SHAPE, "n_nodes must be in 1..%d", kMaxRows);
   if (!t->parent || !t->depth || !t->rank) return fail(nullptr, AMPH_ERR_INVALID_ARG, "tree arrays must not be NULL");
+  if (c->max_batch * round_up(t->n_nodes < 16 ? 16 : t->n_nodes, 16) > kPrefillGroups * kMaxRows)
+    return fail(nullptr, AMPH_ERR_SHAPE, "max_batch * tree nodes (rounded up to 16) must not exceed %d rows", kPrefillGroups * kMaxRows);
   if (c->max_ctx < t->n_nodes + 1) return fail(nullptr, AMPH_ERR_SHAPE, "max_ctx must exceed n_nodes");
   TreeDev td;
   memset(&td, 0, sizeof td);
@@ -184,68 +211,72 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
   return AMPH_OK;
 }
 
-// A prefill chunk carries as many rows as one pass can (every chunk streams all weights once).
-constexpr int kPrefillRows = kMaxRows;
-
-void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, size_t* kv_bytes, int* Mver_out = nullptr) {
+void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, size_t* kv_bytes, int* Mver_out = nullptr,
+                 int* Rcap_out = nullptr, int* small_cap_out = nullptr) {
   const int Mver = round_up(n_nodes < 16 ? 16 : n_nodes, 16);
   const int Mcap = Mver > kPrefillRows ? Mver : kPrefillRows;
+  const int B = c.max_batch;
+  int Rcap = kPrefillGroups * kPrefillRows;                   // a dense prefill pass
+  if (B * Mver > Rcap) Rcap = B * Mver;
+  const int small_cap = round_up(B * (c.K > 2 ? c.K : 2) > B * kSmallRows ? B * c.K : B * kSmallRows, 16);
   if (Mver_out) *Mver_out = Mver;
+  if (Rcap_out) *Rcap_out = Rcap;
+  if (small_cap_out) *small_cap_out = small_cap;
   const size_t esz = c.weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
   const size_t d = c.d_model, F = c.d_ffn, V = c.vocab, half = c.head_dim / 2;
   Layout l;
-  l.state = l.take(sizeof(DevState));
+  l.state = l.per_group(sizeof(DevState), &l.state_s);
+  l.meta_v = l.per_group(sizeof(RowMeta), &l.meta_s_);
+  l.meta_s = l.per_group(sizeof(RowMeta), &l.meta_s_);
+  l.kv_tab = l.per_group(sizeof(KvView) * c.n_layers, &l.kv_tab_s);
+  l.rope_v = l.per_group(sizeof(float2) * Mcap * half, &l.rope_s_);
+  l.rope_s = l.per_group(sizeof(float2) * Mcap * half, &l.rope_s_);
+  l.topk_ids = l.per_group(sizeof(int) * kMaxK * kTopkStride, &l.topk_ids_s);
+  l.topk_vals = l.per_group(sizeof(float) * kMaxK * kTopkStride, &l.topk_vals_s);
+  l.topk_cand = l.per_group(2 * sizeof(float) * kMaxK * kTopkCandChunks * kTopkStride, &l.topk_cand_s);
+  l.last = l.per_group(4 * 2 * d, &l.last_s);
+  l.d_logits = l.per_group(4 * (size_t)kMaxK * V, &l.d_logits_s);
   l.tree = l.take(sizeof(TreeDev));
-  l.meta_v = l.take(sizeof(RowMeta));
-  l.meta_s = l.take(sizeof(RowMeta));
-  l.kv_tab = l.take(sizeof(KvView) * c.n_layers);
   l.inv_freq = l.take(sizeof(double) * half);
-  l.rope_v = l.take(sizeof(float2) * Mcap * half);
-  l.rope_s = l.take(sizeof(float2) * Mcap * half);
-  l.tok = l.take(sizeof(int) * kMaxRows);
-  l.amax = l.take(sizeof(int) * kMaxRows);
-  l.override_tok = l.take(sizeof(int) * kMaxRows);
-  l.next_tok = l.take(sizeof(int) * kMaxRows);
-  l.topk_ids = l.take(sizeof(int) * kMaxK * kTopkStride);
-  l.topk_vals = l.take(sizeof(float) * kMaxK * kTopkStride);
-  l.topk_cand = l.take(2 * sizeof(float) * kMaxK * kTopkCandChunks * kTopkStride);
-  l.amax_cand = l.take(2 * sizeof(float) * kMaxRows * 8);
-  l.x = l.take(4 * Mcap * d);
-  l.hidden = l.take(4 * Mcap * d);
-  l.h1 = l.take(4 * Mcap * d);
-  l.h2 = l.take(4 * Mcap * d);
-  l.pend_h = l.take(4 * 16 * d);
-  l.last = l.take(4 * 2 * d);
-  l.hp = l.take(4 * kMaxK * d);
-  l.attn_o = l.take(4 * 16 * d);
-  l.xn = l.take(esz * Mcap * d);
-  l.q = l.take(esz * Mcap * d);
-  l.att = l.take(esz * Mcap * d);
-  l.act = l.take(esz * Mcap * F);
-  l.cat = l.take(esz * Mcap * 2 * d);
-  l.last_act = l.take(esz * 16 * d);
-  l.ao_act = l.take(esz * 16 * d);
-  l.aeb_act = l.take(esz * 16 * d);
-  l.lr_act = l.take(esz * 16 * (size_t)(c.lm_rank > 0 ? c.lm_rank : 8));
+  l.tok = l.take(sizeof(int) * Rcap);
+  l.amax = l.take(sizeof(int) * Rcap);
+  l.override_tok = l.take(sizeof(int) * Rcap);
+  l.next_tok = l.take(sizeof(int) * Rcap);
+  l.amax_cand = l.take(2 * sizeof(float) * Rcap * 8);
+  l.x = l.take(4 * Rcap * d);
+  l.hidden = l.take(4 * Rcap * d);
+  l.h1 = l.take(4 * Rcap * d);
+  l.h2 = l.take(4 * Rcap * d);
+  l.pend_h = l.take(4 * (size_t)kMaxSeq * kSmallRows * d);     // [sequence][16][d]: the rows of a draft pass back to back
+  l.hp = l.take(4 * (size_t)kMaxSeq * kMaxK * d);               // [sequence][K][d]
+  l.attn_o = l.take(4 * (size_t)small_cap * d);                 // [sequence * K + k][d]
+  l.xn = l.take(esz * Rcap * d);
+  l.q = l.take(esz * Rcap * d);
+  l.att = l.take(esz * Rcap * d);
+  l.act = l.take(esz * Rcap * F);
+  l.cat = l.take(esz * Rcap * 2 * d);
+  l.last_act = l.take(esz * small_cap * d);
+  l.ao_act = l.take(esz * small_cap * d);
+  l.aeb_act = l.take(esz * small_cap * d);
+  l.lr_act = l.take(esz * small_cap * (size_t)(c.lm_rank > 0 ? c.lm_rank : 8));
   size_t big = 3 * d > 2 * F ? 3 * d : 2 * F;
-  size_t pf = 4 * (size_t)Mcap * big;                       // room for 4 K-splits of the widest projection
-  if (2 * (size_t)Mcap * V > pf) pf = 2 * (size_t)Mcap * V;
-  if ((size_t)16 * c.K * V > pf) pf = (size_t)16 * c.K * V;
+  size_t pf = 4 * (size_t)Rcap * big;                       // room for 4 K-splits of the widest projection
+  if (2 * (size_t)Rcap * V > pf) pf = 2 * (size_t)Rcap * V;
+  if ((size_t)small_cap * c.K * V > pf) pf = (size_t)small_cap * c.K * V;
   l.partial_floats = pf;
   l.partial = l.take(4 * pf);
   int splits = (296 + c.n_heads - 1) / c.n_heads;
   if (splits > 8) splits = 8;                               // the KV splits of a head run as one thread-block cluster (<= 8 CTAs)
   l.attn_splits = splits;
-  l.att_o = l.take(4 * (size_t)splits * c.n_heads * Mcap * c.head_dim);
-  l.att_ml = l.take(4 * (size_t)splits * c.n_heads * Mcap * 2);
-  l.logits = l.take(4 * (size_t)Mcap * V);
-  l.d_logits = l.take(4 * (size_t)kMaxK * V);
-  l.ss_a = l.take(4 * (size_t)Mcap * 32);
-  l.ss_b = l.take(4 * (size_t)Mcap * 32);
+  l.att_o = l.per_group(4 * (size_t)splits * c.n_heads * Mcap * c.head_dim, &l.att_o_s);
+  l.att_ml = l.per_group(4 * (size_t)splits * c.n_heads * Mcap * 2, &l.att_ml_s);
+  l.logits = l.take(4 * (size_t)Rcap * V);
+  l.ss_a = l.take(4 * (size_t)Rcap * 32);
+  l.ss_b = l.take(4 * (size_t)Rcap * 32);
   *L = l;
   *Mcap_out = Mcap;
   const size_t per_layer = 2 * (size_t)c.n_heads * c.max_ctx * c.head_dim * esz;
-  *kv_bytes = per_layer * (c.n_layers + c.n_sal);
+  *kv_bytes = per_layer * (c.n_layers + c.n_sal) * B;
 }
 
 // ---- weights ------------------------------------------------------------------------------
@@ -368,62 +399,99 @@ RowScale row_scale_of(const amph_ctx* ctx, size_t off) {
   return rs;
 }
 
-// One decoder layer over the rows described by `meta`.
+// A forward pass: G row groups of rpg rows each.  Group g uses row table meta[g], rotary table rope[g], the caches of
+// sequence seq[g], and may see at most keys[g] cache slots (host-side bound: committed slots + the rows of the pass).
+struct Pass {
+  int G = 1;
+  int rpg = 0;
+  const RowMeta* meta[kMaxSeq];
+  float2* rope[kMaxSeq];
+  int seq[kMaxSeq];
+  int keys[kMaxSeq];
+  int rows() const { return G * rpg; }
+};
+
+PartialView rows_from(PartialView P, int row0) {
+  P.p += (size_t)row0 * P.ld;
+  return P;
+}
+RowScale rows_from(RowScale rs, int row0) {
+  if (rs.ss) rs.ss += (size_t)row0 * rs.chunks;
+  return rs;
+}
+
+void pass_rope_tables(amph_ctx* ctx, const Pass& ps) {
+  for (int g = 0; g < ps.G; ++g) {
+    ProfScope p(ctx, AMPH_PROF_OTHER);
+    launch_rope_table(ps.meta[g], ctx->at<double>(ctx->lay.inv_freq), ps.rope[g], ps.rpg, ctx->cfg.head_dim / 2, ctx->stream);
+  }
+}
+
+// One decoder layer over the rows of the pass; cache_of(seq) gives the layer's cache of a sequence.
 // Entry: xn holds the input of the q/k/v projections: attn_norm * x / rms(x) if !entry_deferred, else
 // attn_norm * x with the row sums of squares in ss_a (the division is applied after the projection).
 // Exit: x is updated.  With next_gain and no hid: xn = next_gain * x, sums of squares in ss_a (deferred form
 // for the next layer; returns true).  With hid: xn and hid hold the normalised rows (returns false).
-bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const RowMeta* meta, const float2* rope,
-                   int rows, int ctx_hi, const void* next_gain, float* hid, bool entry_deferred) {
+template <typename CacheOf>
+bool layer_forward(amph_ctx* ctx, const LayerW& w, CacheOf cache_of, float* x, const Pass& ps, const void* next_gain,
+                   float* hid, bool entry_deferred) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
+  const int rows = ps.rows();
+  const size_t d = c.d_model;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
   PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
-  { ProfScope ps(ctx, AMPH_PROF_ROPE_KV);
-  launch_qkv_rope(P, meta, rope, ctx->ws + l.q, kv, ctx->dtype, rows, c.n_heads, c.head_dim, c.max_ctx, st,
-                  entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale());
+  const RowScale rs = entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale();
+  for (int g = 0; g < ps.G; ++g) {                    // rotary embedding + cache write, per group (its own cache and slots)
+    ProfScope p(ctx, AMPH_PROF_ROPE_KV);
+    launch_qkv_rope(rows_from(P, g * ps.rpg), ps.meta[g], ps.rope[g], ctx->ws + l.q + ctx->esz * g * ps.rpg * d, cache_of(ps.seq[g]),
+                    ctx->dtype, ps.rpg, c.n_heads, c.head_dim, c.max_ctx, st, rows_from(rs, g * ps.rpg));
   }
-  AttnScratch sc = {ctx->at<float>(l.att_o), ctx->at<float>(l.att_ml)};
-  { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
-  bool done = false;
-  if (ctx->attn_tc) {
-    const int splits = attn_tc_splits(ctx->attn_tc, ctx_hi, c.n_heads, rows, l.attn_splits);
-    const bool merged = !(c.flags & AMPH_FLAG_SEPARATE_MERGE);
-    done = launch_tree_attention_tc(ctx->attn_tc, ctx->ws + l.q, ctx->Mcap, kv, meta, sc, rows, c.n_heads, c.head_dim, c.max_ctx,
-                                    splits, ctx_hi, st, merged ? ctx->ws + l.att : nullptr, &ctx->at<DevState>(l.state)->err);
-    if (done && !merged)
-      launch_attn_combine(sc, ctx->ws + l.att, ctx->dtype, splits, rows, c.n_heads, c.head_dim, st, ctx->tc != nullptr);
-    if (!done) cudaGetLastError();
-  }
-  if (!done)
-    launch_tree_attention(ctx->ws + l.q, kv, meta, sc, ctx->ws + l.att, ctx->dtype, rows, c.n_heads, c.head_dim,
-                          c.max_ctx, ctx_hi, l.attn_splits, st, ctx->tc != nullptr,
-                          (c.flags & AMPH_FLAG_SEPARATE_MERGE) != 0);
+  for (int g = 0; g < ps.G; ++g) {                    // tree attention, per group
+    ProfScope p(ctx, AMPH_PROF_ATTENTION);
+    const KvView kv = cache_of(ps.seq[g]);
+    AttnScratch sc = {ctx->grp<float>(l.att_o, l.att_o_s, g), ctx->grp<float>(l.att_ml, l.att_ml_s, g)};
+    char* qg = ctx->ws + l.q + ctx->esz * g * ps.rpg * d;
+    char* og = ctx->ws + l.att + ctx->esz * g * ps.rpg * d;
+    const bool last_g = g + 1 == ps.G;
+    bool done = false;
+    if (ctx->attn_tc) {
+      const int splits = attn_tc_splits(ctx->attn_tc, ps.keys[g], c.n_heads, ps.rpg, l.attn_splits);
+      const bool merged = !(c.flags & AMPH_FLAG_SEPARATE_MERGE);
+      done = launch_tree_attention_tc(ctx->attn_tc, qg, ctx->Rcap - g * ps.rpg, kv, ps.meta[g], sc, ps.rpg, c.n_heads, c.head_dim,
+                                      c.max_ctx, splits, ps.keys[g], st, merged ? og : nullptr, &ctx->state(0)->err);
+      if (done && !merged)
+        launch_attn_combine(sc, og, ctx->dtype, splits, ps.rpg, c.n_heads, c.head_dim, st, last_g && ctx->tc != nullptr);
+      if (!done) cudaGetLastError();
+    }
+    if (!done)
+      launch_tree_attention(qg, kv, ps.meta[g], sc, og, ctx->dtype, ps.rpg, c.n_heads, c.head_dim, c.max_ctx, ps.keys[g],
+                            l.attn_splits, st, last_g && ctx->tc != nullptr, (c.flags & AMPH_FLAG_SEPARATE_MERGE) != 0);
   }
   const void* wo[1] = {w.wo};
   P = project(ctx, XB_ATT, wo, 1, c.d_model, c.d_model, rows);
-  { ProfScope ps(ctx, AMPH_PROF_NORM);
+  { ProfScope p(ctx, AMPH_PROF_NORM);
   launch_resid_scale(x, P, 0, 1, w.ffn_norm, ctx->dtype, ctx->ws + l.xn, ctx->at<float>(l.ss_b), rows, c.d_model, st,
                      ctx->last_proj_one_wave);
   }
   bool fused_gu = false;
   if (ctx->tc && !(c.flags & AMPH_FLAG_SEPARATE_SWIGLU)) {         // gate / up projection with SwiGLU in its epilogue
-    ProfScope ps(ctx, AMPH_PROF_PROJECTION);
+    ProfScope p(ctx, AMPH_PROF_PROJECTION);
     fused_gu = tc_gemm_launch_swiglu(ctx->tc, XB_XN, w.w_gate, w.w_up, c.d_ffn, c.d_model, rows, ctx->ws + l.act,
                                      row_scale_of(ctx, l.ss_b), st);
-    if (fused_gu && ps.rec) ctx->prof_bytes += 2LL * c.d_ffn * c.d_model * (int64_t)ctx->esz;
+    if (fused_gu && p.rec) ctx->prof_bytes += 2LL * c.d_ffn * c.d_model * (int64_t)ctx->esz;
     if (fused_gu) ctx->last_proj_one_wave = false;
   }
   if (!fused_gu) {
     const void* gu[2] = {w.w_gate, w.w_up};
     P = project(ctx, XB_XN, gu, 2, c.d_ffn, c.d_model, rows);
-    ProfScope ps(ctx, AMPH_PROF_SWIGLU);
+    ProfScope p(ctx, AMPH_PROF_SWIGLU);
     launch_swiglu(P, ctx->ws + l.act, ctx->dtype, rows, c.d_ffn, st, row_scale_of(ctx, l.ss_b), ctx->last_proj_one_wave);
   }
   const void* wd[1] = {w.w_down};
   P = project(ctx, XB_ACT, wd, 1, c.d_model, c.d_ffn, rows);
-  ProfScope ps(ctx, AMPH_PROF_NORM);
+  ProfScope p(ctx, AMPH_PROF_NORM);
   if (hid != nullptr) {
     launch_resid_norm(x, P, 0, 1, next_gain, ctx->dtype, ctx->ws + l.xn, hid, c.rms_eps, rows, c.d_model, st);
     return false;
@@ -433,29 +501,26 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, KvView kv, float* x, const Ro
   return next_gain != nullptr;
 }
 
-// Target forward of the rows in `tok` under meta_v; leaves post-final-norm rows in hidden and xn.
-void target_forward(amph_ctx* ctx, int rows, int ctx_hi) {
+// Target forward of the tokens in `tok` (one per row of the pass); leaves post-final-norm rows in hidden and xn.
+void target_forward(amph_ctx* ctx, const Pass& ps) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const RowMeta* meta = ctx->at<RowMeta>(l.meta_v);
-  float2* rope = ctx->at<float2>(l.rope_v);
+  const int rows = ps.rows();
   float* x = ctx->at<float>(l.x);
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
-  }
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
+  pass_rope_tables(ctx, ps);
+  { ProfScope p(ctx, AMPH_PROF_OTHER);
   launch_embed(ctx->tok_emb, ctx->dtype, ctx->at<int>(l.tok), c.vocab, rows, c.d_model, x, st);
   }
   PartialView none = {nullptr, 0, 0, 0};
-  { ProfScope ps(ctx, AMPH_PROF_NORM);
+  { ProfScope p(ctx, AMPH_PROF_NORM);
   launch_resid_norm(x, none, 0, 0, ctx->layers[0].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                     c.d_model, st);
   }
   bool deferred = false;
   for (int i = 0; i < c.n_layers; ++i) {
     const bool last = i + 1 == c.n_layers;
-    deferred = layer_forward(ctx, ctx->layers[i], ctx->kv_target[i], x, meta, rope, rows, ctx_hi,
+    deferred = layer_forward(ctx, ctx->layers[i], [&](int b) { return ctx->kv_target[b][i]; }, x, ps,
                              last ? ctx->final_norm : ctx->layers[i + 1].attn_norm,
                              last ? ctx->at<float>(l.hidden) : nullptr, deferred);
   }
@@ -466,35 +531,36 @@ void target_head(amph_ctx* ctx, int rows) {
   const Layout& l = ctx->lay;
   const void* w[1] = {ctx->lm_head};
   PartialView P = project(ctx, XB_XN, w, 1, c.vocab, c.d_model, rows);
-  { ProfScope ps(ctx, AMPH_PROF_SELECT);
+  { ProfScope p(ctx, AMPH_PROF_SELECT);
   launch_argmax_rows(P, c.vocab, rows, ctx->at<int>(l.amax), ctx->at<float>(l.logits), ctx->at<float>(l.amax_cand), ctx->stream);
   }
 }
 
-// Eq. 1: both adaptation stages over the rows (feat, next_tok) described by meta_s.
-void run_sals(amph_ctx* ctx, const float* feat, const int* next_tok, int rows, int ctx_hi) {
+// Eq. 1: both adaptation stages over the rows of the pass.  feat: fp32 rows [rows][d]; next_tok[g]: the ids of the
+// tokens that follow group g's rows (rpg entries).
+void run_sals(amph_ctx* ctx, const float* feat, const int* const* next_tok, const Pass& ps) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const RowMeta* meta = ctx->at<RowMeta>(l.meta_s);
-  float2* rope = ctx->at<float2>(l.rope_s);
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_rope_table(meta, ctx->at<double>(l.inv_freq), rope, rows, c.head_dim / 2, st);
-  }
+  const int rows = ps.rows();
+  const bool with_tok = !(c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN);             // Section 4.5, "w/o Sampled-Token"
+  const size_t cat_pitch = (with_tok ? 2 : 1) * (size_t)c.d_model * ctx->esz;
+  pass_rope_tables(ctx, ps);
   const float* in_feat = feat;
   for (int s = 0; s < c.n_sal; ++s) {
     float* hbuf = ctx->at<float>(s == 0 ? l.h1 : l.h2);
-    { ProfScope ps(ctx, AMPH_PROF_OTHER);
-    const bool with_tok = !(c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN);             // Section 4.5, "w/o Sampled-Token"
-    launch_concat(in_feat, with_tok ? ctx->tok_emb : nullptr, next_tok, c.vocab, ctx->ws + l.cat, ctx->dtype, rows, c.d_model, st);
+    for (int g = 0; g < ps.G; ++g) {
+      ProfScope p(ctx, AMPH_PROF_OTHER);
+      launch_concat(in_feat + (size_t)g * ps.rpg * c.d_model, with_tok ? ctx->tok_emb : nullptr, next_tok[g], c.vocab,
+                    ctx->ws + l.cat + cat_pitch * g * ps.rpg, ctx->dtype, ps.rpg, c.d_model, st);
     }
     const void* w[1] = {ctx->fc[s]};
-    PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, ((c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN) ? 1 : 2) * c.d_model, rows);
-    { ProfScope ps(ctx, AMPH_PROF_NORM);
+    PartialView P = project(ctx, XB_CAT, w, 1, c.d_model, (with_tok ? 2 : 1) * c.d_model, rows);
+    { ProfScope p(ctx, AMPH_PROF_NORM);
     launch_resid_norm(hbuf, P, 0, 2, ctx->sal[s].attn_norm, ctx->dtype, ctx->ws + l.xn, nullptr, c.rms_eps, rows,
                       c.d_model, st);
     }
-    layer_forward(ctx, ctx->sal[s], ctx->kv_sal[s], hbuf, meta, rope, rows, ctx_hi, nullptr, nullptr, false);
+    layer_forward(ctx, ctx->sal[s], [&](int b) { return ctx->kv_sal[b][s]; }, hbuf, ps, nullptr, nullptr, false);
     in_feat = hbuf;
   }
 }
@@ -507,104 +573,148 @@ amph_status copy_out(amph_ctx* ctx, void* dst, const void* src, size_t bytes) {
 amph_status finish(amph_ctx* ctx, const char* what) { return cuda_check(ctx, cudaGetLastError(), what); }
 
 amph_status refresh_ctx_hi(amph_ctx* ctx) {
-  DevState s;
-  cudaError_t e = cudaMemcpyAsync(&s, ctx->at<DevState>(ctx->lay.state), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
-  if (e != cudaSuccess) return cuda_check(ctx, e, "state read-back");
-  ctx->ctx_hi = s.C;
-  if (s.err) return fail(ctx, s.err, "a device-side wait gave up (code %d)", s.err);
+  for (int b = 0; b < ctx->B; ++b) {
+    if (!ctx->prefilled[b]) continue;
+    DevState s;
+    cudaError_t e = cudaMemcpyAsync(&s, ctx->state(b), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) return cuda_check(ctx, e, "state read-back");
+    ctx->ctx_hi[b] = s.C;
+    if (s.err) return fail(ctx, s.err, "a device-side wait gave up (code %d)", s.err);
+  }
   return AMPH_OK;
 }
 
+// out_ids / out_vals: [B][K][AMPH_TOPK_STRIDE]
 amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  DevState* ds = ctx->at<DevState>(l.state);
-  const int rows = ctx->rows_small;
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_meta_pending(ctx->at<RowMeta>(l.meta_s), ds, st);
+  const int B = ctx->B, K = c.K;
+  const size_t d = c.d_model;
+  Pass ps;
+  ps.G = B;
+  ps.rpg = ctx->rows_small;
+  const int* next_tok[kMaxSeq];
+  for (int b = 0; b < B; ++b) {
+    ps.meta[b] = ctx->meta_s(b);
+    ps.rope[b] = ctx->grp<float2>(l.rope_s, l.rope_s_, b);
+    ps.seq[b] = b;
+    ps.keys[b] = ctx->ctx_hi[b];
+    next_tok[b] = ctx->state(b)->pend_tok;
+    ProfScope p(ctx, AMPH_PROF_OTHER);
+    launch_meta_pending(ctx->meta_s(b), ctx->state(b), st);
   }
-  run_sals(ctx, ctx->at<float>(l.pend_h), ds->pend_tok, rows, ctx->ctx_hi);
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
+  float* pend_h = ctx->at<float>(l.pend_h);            // [B][16][d] = the rows of this pass
+  run_sals(ctx, pend_h, next_tok, ps);
   // without adaptation layers (the "w/o Staged-Adaptation" ablation) every head reads the target's hidden state itself
-  const float* s1 = ctx->at<float>(c.n_sal == 0 ? l.pend_h : l.h1);
-  const float* s2 = ctx->at<float>(c.n_sal == 0 ? l.pend_h : (c.n_sal == 2 ? l.h2 : l.h1));
-  launch_gather_last(s1, s2, ds, ctx->at<float>(l.last), ctx->ws + l.last_act, ctx->dtype, c.d_model, st);
+  const float* s1 = c.n_sal == 0 ? pend_h : ctx->at<float>(l.h1);
+  const float* s2 = c.n_sal == 0 ? pend_h : ctx->at<float>(c.n_sal == 2 ? l.h2 : l.h1);
+  for (int b = 0; b < B; ++b) {                        // rows 2 b, 2 b + 1 of the head MLPs' input: the last row of each stage
+    ProfScope p(ctx, AMPH_PROF_OTHER);
+    launch_gather_last(s1 + (size_t)b * ps.rpg * d, s2 + (size_t)b * ps.rpg * d, ctx->state(b), ctx->grp<float>(l.last, l.last_s, b),
+                       ctx->ws + l.last_act + ctx->esz * 2 * b * d, ctx->dtype, c.d_model, st);
   }
-  PartialView P = project(ctx, XB_LAST, ctx->mlp_w, c.K, c.d_model, c.d_model, 2);                   // Eq. 2
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_mlp_heads(P, ctx->at<float>(l.last), ctx->mlp_b, ctx->pe, ctx->at<float>(l.hp), ctx->at<float>(l.attn_o),
-                   ctx->ws + l.ao_act, ctx->dtype, c.K, c.n_sal, c.d_model, st);                      // Eq. 3-4
+  PartialView P = project(ctx, XB_LAST, ctx->mlp_w, K, c.d_model, c.d_model, 2 * B);                 // Eq. 2
+  float* hp = ctx->at<float>(l.hp);
+  float* ao = ctx->at<float>(l.attn_o);
+  for (int b = 0; b < B; ++b) {                                                                       // Eq. 3-4
+    ProfScope p(ctx, AMPH_PROF_OTHER);
+    launch_mlp_heads(rows_from(P, 2 * b), ctx->grp<float>(l.last, l.last_s, b), ctx->mlp_b, ctx->pe, hp + (size_t)b * kMaxK * d,
+                     ao + (size_t)b * K * d, ctx->ws + l.ao_act + ctx->esz * b * K * d, ctx->dtype, K, c.n_sal, c.d_model, st);
   }
   for (int a = 0; a < c.aeb_layers; ++a) {                                                            // Eq. 5
-    P = project(ctx, XB_AO, ctx->aeb_w[a], 3, c.d_model, c.d_model, c.K);
-    { ProfScope ps(ctx, AMPH_PROF_ATTENTION);
-    launch_aeb_attention(P, ctx->ws + l.aeb_act, ctx->dtype, c.K, c.n_heads, c.head_dim, st);
+    P = project(ctx, XB_AO, ctx->aeb_w[a], 3, c.d_model, c.d_model, B * K);
+    for (int b = 0; b < B; ++b) {                       // the K rows of a sequence attend to each other only
+      ProfScope p(ctx, AMPH_PROF_ATTENTION);
+      launch_aeb_attention(rows_from(P, b * K), ctx->ws + l.aeb_act + ctx->esz * b * K * d, ctx->dtype, K, c.n_heads, c.head_dim, st);
     }
     const void* wo[1] = {ctx->aeb_w[a][3]};
-    P = project(ctx, XB_AEB, wo, 1, c.d_model, c.d_model, c.K);
-    { ProfScope ps(ctx, AMPH_PROF_NORM);
-    launch_resid_norm(ctx->at<float>(l.attn_o), P, 0, 1, nullptr, ctx->dtype, ctx->ws + l.ao_act, nullptr, c.rms_eps,
-                      c.K, c.d_model, st);
+    P = project(ctx, XB_AEB, wo, 1, c.d_model, c.d_model, B * K);
+    { ProfScope p(ctx, AMPH_PROF_NORM);
+    launch_resid_norm(ao, P, 0, 1, nullptr, ctx->dtype, ctx->ws + l.ao_act, nullptr, c.rms_eps, B * K, c.d_model, st);
     }
   }
   if (c.lm_rank > 0) {                                                                                // Appendix A.2.4
-    P = project(ctx, XB_AO, ctx->draft_lm_a, c.K, c.lm_rank, c.d_model, c.K);
-    { ProfScope ps(ctx, AMPH_PROF_OTHER);
-    launch_gather_diag(P, ctx->ws + l.lr_act, ctx->dtype, c.K, c.lm_rank, st);
+    P = project(ctx, XB_AO, ctx->draft_lm_a, K, c.lm_rank, c.d_model, B * K);
+    for (int b = 0; b < B; ++b) {
+      ProfScope p(ctx, AMPH_PROF_OTHER);
+      launch_gather_diag(rows_from(P, b * K), ctx->ws + l.lr_act + ctx->esz * b * K * (size_t)c.lm_rank, ctx->dtype, K, c.lm_rank, st);
     }
-    P = project(ctx, XB_LR, ctx->draft_lm, c.K, c.vocab, c.lm_rank, c.K);
+    P = project(ctx, XB_LR, ctx->draft_lm, K, c.vocab, c.lm_rank, B * K);
   } else {
-    P = project(ctx, XB_AO, ctx->draft_lm, c.K, c.vocab, c.d_model, c.K);                             // Eq. 6
+    P = project(ctx, XB_AO, ctx->draft_lm, K, c.vocab, c.d_model, B * K);                             // Eq. 6
   }
-  { ProfScope ps(ctx, AMPH_PROF_SELECT);
-  launch_topk_heads(P, c.vocab, c.K, c.topk, ctx->at<int>(l.topk_ids), ctx->at<float>(l.topk_vals),
-                    ctx->at<float>(l.d_logits), ctx->at<float>(l.topk_cand), st);
+  for (int b = 0; b < B; ++b) {
+    { ProfScope p(ctx, AMPH_PROF_SELECT);
+    launch_topk_heads(rows_from(P, b * K), c.vocab, K, c.topk, ctx->grp<int>(l.topk_ids, l.topk_ids_s, b),
+                      ctx->grp<float>(l.topk_vals, l.topk_vals_s, b), ctx->grp<float>(l.d_logits, l.d_logits_s, b),
+                      ctx->grp<float>(l.topk_cand, l.topk_cand_s, b), st);
+    }
+    { ProfScope p(ctx, AMPH_PROF_OTHER);
+    launch_tree_build(ctx->at<TreeDev>(l.tree), ctx->state(b), ctx->grp<int>(l.topk_ids, l.topk_ids_s, b), nullptr,
+                      ctx->at<int>(l.tok) + b * ctx->Mver, ctx->meta_v(b), st);
+    }
   }
-  { ProfScope ps(ctx, AMPH_PROF_OTHER);
-  launch_tree_build(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.topk_ids), nullptr, ctx->at<int>(l.tok),
-                    ctx->at<RowMeta>(l.meta_v), st);
+  amph_status rc = AMPH_OK;
+  for (int b = 0; b < B && rc == AMPH_OK; ++b) {
+    if (out_ids) rc = copy_out(ctx, out_ids + (size_t)b * K * kTopkStride, ctx->grp<int>(l.topk_ids, l.topk_ids_s, b), sizeof(int) * K * kTopkStride);
+    if (rc == AMPH_OK && out_vals)
+      rc = copy_out(ctx, out_vals + (size_t)b * K * kTopkStride, ctx->grp<float>(l.topk_vals, l.topk_vals_s, b), sizeof(float) * K * kTopkStride);
   }
-  amph_status rc = copy_out(ctx, out_ids, ctx->at<int>(l.topk_ids), sizeof(int) * c.K * kTopkStride);
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_vals, ctx->at<float>(l.topk_vals), sizeof(float) * c.K * kTopkStride);
   return rc;
 }
 
+// tree_tokens / out_argmax: [B][n_nodes]
 amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_argmax) {
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const int N = ctx->tree_host.n_nodes;
-  if (tree_tokens) {
-    amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.override_tok), tree_tokens, sizeof(int) * N,
-                                                     cudaMemcpyDefault, st), "copy of tree tokens");
-    if (rc != AMPH_OK) return rc;
-    { ProfScope ps(ctx, AMPH_PROF_OTHER);
-    launch_tree_build(ctx->at<TreeDev>(l.tree), ctx->at<DevState>(l.state), nullptr, ctx->at<int>(l.override_tok),
-                      ctx->at<int>(l.tok), ctx->at<RowMeta>(l.meta_v), st);
+  const int N = ctx->tree_host.n_nodes, B = ctx->B;
+  Pass ps;
+  ps.G = B;
+  ps.rpg = ctx->Mver;
+  for (int b = 0; b < B; ++b) {
+    ps.meta[b] = ctx->meta_v(b);
+    ps.rope[b] = ctx->grp<float2>(l.rope_v, l.rope_s_, b);
+    ps.seq[b] = b;
+    ps.keys[b] = ctx->ctx_hi[b] + N;
+    if (tree_tokens) {
+      int* ov = ctx->at<int>(l.override_tok) + b * ctx->Mver;
+      amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ov, tree_tokens + (size_t)b * N, sizeof(int) * N, cudaMemcpyDefault, st), "copy of tree tokens");
+      if (rc != AMPH_OK) return rc;
+      ProfScope p(ctx, AMPH_PROF_OTHER);
+      launch_tree_build(ctx->at<TreeDev>(l.tree), ctx->state(b), nullptr, ov, ctx->at<int>(l.tok) + b * ctx->Mver, ctx->meta_v(b), st);
     }
   }
-  target_forward(ctx, ctx->Mver, ctx->ctx_hi + N);
-  target_head(ctx, ctx->Mver);
-  return copy_out(ctx, out_argmax, ctx->at<int>(l.amax), sizeof(int) * N);
+  target_forward(ctx, ps);
+  target_head(ctx, ps.rows());
+  amph_status rc = AMPH_OK;
+  for (int b = 0; b < B && rc == AMPH_OK && out_argmax; ++b)
+    rc = copy_out(ctx, out_argmax + (size_t)b * N, ctx->at<int>(l.amax) + b * ctx->Mver, sizeof(int) * N);
+  return rc;
 }
 
+// out_tokens, out_path: [B][K+1]; out_n, out_next_root: [B]
 amph_status do_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_t* out_path, int32_t* out_next_root) {
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  DevState* ds = ctx->at<DevState>(l.state);
-  { ProfScope ps(ctx, AMPH_PROF_ACCEPT);
-  launch_accept(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.tok), ctx->at<int>(l.amax), st);
+  amph_status rc = AMPH_OK;
+  for (int b = 0; b < ctx->B && rc == AMPH_OK; ++b) {
+    DevState* ds = ctx->state(b);
+    { ProfScope p(ctx, AMPH_PROF_ACCEPT);
+    launch_accept(ctx->at<TreeDev>(l.tree), ds, ctx->at<int>(l.tok) + b * ctx->Mver, ctx->at<int>(l.amax) + b * ctx->Mver, st);
+    }
+    { ProfScope p(ctx, AMPH_PROF_ACCEPT);
+    launch_compact(ds, ctx->grp<KvView>(l.kv_tab, l.kv_tab_s, b), c.n_layers, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx,
+                   ctx->at<float>(l.hidden) + (size_t)b * ctx->Mver * c.d_model,
+                   ctx->at<float>(l.pend_h) + (size_t)b * kSmallRows * c.d_model, c.d_model, st);
+    }
+    if (out_tokens) rc = copy_out(ctx, out_tokens + b * (c.K + 1), ds->out_tok, sizeof(int) * (c.K + 1));
+    if (rc == AMPH_OK && out_n) rc = copy_out(ctx, out_n + b, &ds->L, sizeof(int));
+    if (rc == AMPH_OK && out_path) rc = copy_out(ctx, out_path + b * (c.K + 1), ds->path, sizeof(int) * (c.K + 1));
+    if (rc == AMPH_OK && out_next_root) rc = copy_out(ctx, out_next_root + b, &ds->next_root, sizeof(int));
   }
-  { ProfScope ps(ctx, AMPH_PROF_ACCEPT);
-  launch_compact(ds, ctx->at<KvView>(l.kv_tab), c.n_layers, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx,
-                 ctx->at<float>(l.hidden), ctx->at<float>(l.pend_h), c.d_model, st);
-  }
-  amph_status rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_path, ds->path, sizeof(int) * (c.K + 1));
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_next_root, &ds->next_root, sizeof(int));
   return rc;
 }
 
@@ -620,13 +730,22 @@ int attn_splits_for(const amph_ctx* ctx, int ctx_hi, int rows) {
 
 amph_status check_capacity(amph_ctx* ctx) {
   const int N = ctx->tree_host.n_nodes;
-  if (ctx->ctx_hi + N > ctx->cfg.max_ctx) {
+  if (ctx->max_ctx_hi() + N > ctx->cfg.max_ctx) {
     amph_status rc = refresh_ctx_hi(ctx);
     if (rc != AMPH_OK) return rc;
-    if (ctx->ctx_hi + N > ctx->cfg.max_ctx)
-      return fail(ctx, AMPH_ERR_CAPACITY, "ctx_len %d + %d tree nodes exceeds max_ctx %d", ctx->ctx_hi, N, ctx->cfg.max_ctx);
+    if (ctx->max_ctx_hi() + N > ctx->cfg.max_ctx)
+      return fail(ctx, AMPH_ERR_CAPACITY, "ctx_len %d + %d tree nodes exceeds max_ctx %d", ctx->max_ctx_hi(), N, ctx->cfg.max_ctx);
   }
   return AMPH_OK;
+}
+
+// The captured schedule depends on the host's bounds only through the attention launches of every sequence.
+long long graph_key_of(const amph_ctx* ctx) {
+  long long key = 0;
+  for (int b = 0; b < ctx->B; ++b)
+    key = key * 4099 + attn_splits_for(ctx, ctx->ctx_hi[b], ctx->rows_small) * 128 +
+          attn_splits_for(ctx, ctx->ctx_hi[b] + ctx->tree_host.n_nodes, ctx->Mver);
+  return key;
 }
 
 }  // namespace
@@ -657,9 +776,9 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   if (!kv_dev || !ws_dev) return fail(nullptr, AMPH_ERR_INVALID_ARG, "kv_dev and ws_dev must not be NULL");
   if (((uintptr_t)kv_dev | (uintptr_t)ws_dev) & 255) return fail(nullptr, AMPH_ERR_WORKSPACE, "regions must be 256-byte aligned");
   Layout l;
-  int Mcap, Mver;
+  int Mcap, Mver, Rcap, small_cap;
   size_t need_kv;
-  make_layout(*cfg, tree->n_nodes, &l, &Mcap, &need_kv, &Mver);
+  make_layout(*cfg, tree->n_nodes, &l, &Mcap, &need_kv, &Mver, &Rcap, &small_cap);
   if (kv_bytes < need_kv) return fail(nullptr, AMPH_ERR_WORKSPACE, "kv region: %zu bytes given, %zu needed", kv_bytes, need_kv);
   if (ws_bytes < l.total) return fail(nullptr, AMPH_ERR_WORKSPACE, "workspace: %zu bytes given, %zu needed", ws_bytes, l.total);
   int dev_count = 0;
@@ -673,22 +792,26 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   ctx->stream = (cudaStream_t)stream;
   ctx->dtype = cfg->weight_dtype;
   ctx->esz = cfg->weight_dtype == AMPH_DTYPE_F32 ? 4 : 2;
+  ctx->B = cfg->max_batch;
   ctx->Mcap = Mcap;
+  ctx->Rcap = Rcap;
   ctx->Mver = Mver;
-  ctx->rows_small = 16;
+  ctx->rows_small = kSmallRows;
+  ctx->small_cap = small_cap;
   ctx->lay = l;
   ctx->ws = (char*)ws_dev;
   ctx->kv = (char*)kv_dev;
   ctx->resolved = false;
   ctx->phase = PH_CREATED;
-  ctx->ctx_hi = 0;
   ctx->tc = nullptr;
   { int dv = 0; cudaGetDevice(&dv); cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dv); }
   const size_t half_layer = (size_t)cfg->n_heads * cfg->max_ctx * cfg->head_dim * ctx->esz;
-  ctx->kv_target.resize(cfg->n_layers);
   char* p = ctx->kv;
-  for (int i = 0; i < cfg->n_layers; ++i) { ctx->kv_target[i].k = p; ctx->kv_target[i].v = p + half_layer; p += 2 * half_layer; }
-  for (int s = 0; s < cfg->n_sal; ++s) { ctx->kv_sal[s].k = p; ctx->kv_sal[s].v = p + half_layer; p += 2 * half_layer; }
+  for (int b = 0; b < ctx->B; ++b) {                   // sequence by sequence: target layers, then the adaptation layers
+    ctx->kv_target[b].resize(cfg->n_layers);
+    for (int i = 0; i < cfg->n_layers; ++i) { ctx->kv_target[b][i].k = p; ctx->kv_target[b][i].v = p + half_layer; p += 2 * half_layer; }
+    for (int s = 0; s < cfg->n_sal; ++s) { ctx->kv_sal[b][s].k = p; ctx->kv_sal[b][s].v = p + half_layer; p += 2 * half_layer; }
+  }
   cudaStream_t st = ctx->stream;
   cudaError_t e = cudaMemsetAsync(ctx->ws, 0, l.total, st);
   // The attention kernels fetch whole key tiles; slots past the live range are masked (probability 0), which only
@@ -697,7 +820,8 @@ amph_status amph_init(const amph_config* cfg, const amph_tree* tree, void* kv_de
   std::vector<double> inv(cfg->head_dim / 2);
   for (int i = 0; i < cfg->head_dim / 2; ++i) inv[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.tree, &ctx->tree_host, sizeof(TreeDev), cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.kv_tab, ctx->kv_target.data(), sizeof(KvView) * cfg->n_layers, cudaMemcpyHostToDevice, st);
+  for (int b = 0; b < ctx->B && e == cudaSuccess; ++b)
+    e = cudaMemcpyAsync(ctx->ws + l.kv_tab + l.kv_tab_s * b, ctx->kv_target[b].data(), sizeof(KvView) * cfg->n_layers, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + l.inv_freq, inv.data(), sizeof(double) * inv.size(), cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) {
@@ -734,9 +858,11 @@ amph_status amph_load_weights(amph_ctx* ctx, const amph_tensor* tensors, int32_t
   return AMPH_OK;
 }
 
-amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, int32_t* out_root) {
+amph_status amph_prefill_seq(amph_ctx* ctx, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* out_root) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (seq < 0 || seq >= ctx->B) return fail(ctx, AMPH_ERR_INVALID_ARG, "sequence %d is outside 0..%d", seq, ctx->B - 1);
   if (!prompt_ids || n < 1) return fail(ctx, AMPH_ERR_INVALID_ARG, "prompt must hold at least one token");
+  if (ctx->phase == PH_DRAFTED || ctx->phase == PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_prefill while a draft is in flight");
   const amph_config& c = ctx->cfg;
   for (int i = 0; i < n; ++i)
     if (prompt_ids[i] < 0 || prompt_ids[i] >= c.vocab) return fail(ctx, AMPH_ERR_INVALID_ARG, "prompt_ids[%d] = %d is outside the vocabulary", i, prompt_ids[i]);
@@ -746,49 +872,85 @@ amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, in
   if (!ctx->tc && c.weight_dtype == AMPH_DTYPE_BF16 && !(c.flags & AMPH_FLAG_NO_TENSOR_CORE)) {
     void* xb[XB_COUNT];
     for (int i = 0; i < XB_COUNT; ++i) xb[i] = xbuf_ptr(ctx, i);
-    const int xrows[XB_COUNT] = {ctx->Mcap, ctx->Mcap, ctx->Mcap, ctx->Mcap, 16, 16, 16, 16};
+    const int sc = ctx->small_cap;
+    const int xrows[XB_COUNT] = {ctx->Rcap, ctx->Rcap, ctx->Rcap, ctx->Rcap, sc, sc, sc, sc};
     const int xcols[XB_COUNT] = {c.d_model, c.d_model, c.d_ffn, ((c.flags & AMPH_FLAG_NO_SAMPLED_TOKEN) ? 1 : 2) * c.d_model,
                                  c.d_model, c.d_model, c.d_model,
                                  c.lm_rank > 0 ? c.lm_rank : 8};
-    ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->at<DevState>(ctx->lay.state)->err);
+    ctx->tc = tc_gemm_create(xb, xrows, xcols, XB_COUNT, &ctx->state(0)->err);
   }
   if (!ctx->attn_tc && c.kv_dtype == AMPH_DTYPE_BF16 && !(c.flags & AMPH_FLAG_MMA_SYNC_ATTENTION))
     ctx->attn_tc = attn_tc_create();
   const Layout& l = ctx->lay;
   cudaStream_t st = ctx->stream;
-  const int M = ctx->Mcap;
-  cudaMemsetAsync(ctx->ws + l.state, 0, sizeof(DevState), st);
-  for (int start = 0; start < n; start += M) {
-    const int nr = n - start < M ? n - start : M;
-    const bool last = start + nr == n;
-    rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.tok), prompt_ids + start, sizeof(int) * nr, cudaMemcpyHostToDevice, st), "prompt upload");
+  const int M = kPrefillRows;
+  // A pass carries up to kPrefillGroups chunks of 128 prompt tokens as row groups that share every weight tile: the
+  // rows of chunk g see the committed slots plus the chunks before them, whose keys and values the same pass has
+  // written by the time attention runs, and a causal mask inside the chunk.
+  const int Gmax = (c.flags & AMPH_FLAG_CHUNKED_PREFILL) ? 1 : kPrefillGroups;
+  cudaMemsetAsync(ctx->state(seq), 0, sizeof(DevState), st);
+  ctx->prefilled[seq] = false;
+  for (int start = 0; start < n; start += Gmax * M) {
+    const int cnt = n - start < Gmax * M ? n - start : Gmax * M;
+    const bool last = start + cnt == n;
+    const int G = (cnt + M - 1) / M;
+    const int rpg = G == 1 ? round_up(cnt, 16) : M;          // rows the kernels carry per group
+    rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.tok), prompt_ids + start, sizeof(int) * cnt, cudaMemcpyHostToDevice, st), "prompt upload");
     if (rc != AMPH_OK) return rc;
-    launch_meta_chain(ctx->at<RowMeta>(l.meta_v), start, nr, st);
-    const int rows = round_up(nr, 16);           // rows the kernels carry for this chunk
-    target_forward(ctx, rows, start + nr);
-    if (last) target_head(ctx, rows);
-    const int nrs = last ? nr - 1 : nr;           // the last prompt row stays pending for the first draft
+    Pass ps;
+    ps.G = G;
+    ps.rpg = rpg;
+    for (int g = 0; g < G; ++g) {
+      const int nr = cnt - g * M < M ? cnt - g * M : M;
+      launch_meta_chain(ctx->meta_v(g), start + g * M, nr, st);
+      ps.meta[g] = ctx->meta_v(g);
+      ps.rope[g] = ctx->grp<float2>(l.rope_v, l.rope_s_, g);
+      ps.seq[g] = seq;
+      ps.keys[g] = start + g * M + nr;
+    }
+    target_forward(ctx, ps);
+    if (last) target_head(ctx, ps.rows());
+    const int nrs = last ? cnt - 1 : cnt;         // the last prompt row stays pending for the first draft
     if (nrs > 0 && c.n_sal > 0) {
       rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<int>(l.next_tok), prompt_ids + start + 1, sizeof(int) * nrs, cudaMemcpyHostToDevice, st), "prompt upload");
       if (rc != AMPH_OK) return rc;
-      launch_meta_chain(ctx->at<RowMeta>(l.meta_s), start, nrs, st);
-      run_sals(ctx, ctx->at<float>(l.hidden), ctx->at<int>(l.next_tok), rows, start + nrs);
+      Pass pss;
+      pss.G = (nrs + M - 1) / M;
+      pss.rpg = rpg;
+      const int* next_tok[kMaxSeq];
+      for (int g = 0; g < pss.G; ++g) {
+        const int nr = nrs - g * M < M ? nrs - g * M : M;
+        launch_meta_chain(ctx->meta_s(g), start + g * M, nr, st);
+        pss.meta[g] = ctx->meta_s(g);
+        pss.rope[g] = ctx->grp<float2>(l.rope_s, l.rope_s_, g);
+        pss.seq[g] = seq;
+        pss.keys[g] = start + g * M + nr;
+        next_tok[g] = ctx->at<int>(l.next_tok) + g * rpg;
+      }
+      run_sals(ctx, ctx->at<float>(l.hidden), next_tok, pss);
     }
     if (last)
-      launch_prefill_tail(ctx->at<DevState>(l.state), ctx->at<int>(l.amax), nr - 1, ctx->at<float>(l.hidden),
-                          ctx->at<float>(l.pend_h), c.d_model, n, st);
+      launch_prefill_tail(ctx->state(seq), ctx->at<int>(l.amax), cnt - 1, ctx->at<float>(l.hidden),
+                          ctx->at<float>(l.pend_h) + (size_t)seq * kSmallRows * c.d_model, c.d_model, n, st);
   }
   rc = finish(ctx, "prefill");
   if (rc != AMPH_OK) return rc;
+  ctx->prefilled[seq] = true;
   rc = refresh_ctx_hi(ctx);
   if (rc != AMPH_OK) return rc;
   if (out_root) {
     DevState s;
-    cudaMemcpy(&s, ctx->at<DevState>(l.state), sizeof s, cudaMemcpyDeviceToHost);
+    cudaMemcpy(&s, ctx->state(seq), sizeof s, cudaMemcpyDeviceToHost);
     *out_root = s.root;
   }
-  ctx->phase = PH_READY;
+  bool all = true;
+  for (int b = 0; b < ctx->B; ++b) all = all && ctx->prefilled[b];
+  ctx->phase = all ? PH_READY : PH_CREATED;
   return AMPH_OK;
+}
+
+amph_status amph_prefill(amph_ctx* ctx, const int32_t* prompt_ids, int32_t n, int32_t* out_root) {
+  return amph_prefill_seq(ctx, 0, prompt_ids, n, out_root);
 }
 
 amph_status amph_draft(amph_ctx* ctx, int32_t* out_topk_ids, float* out_topk_vals) {
@@ -816,7 +978,10 @@ amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int3
   if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_accept must follow amph_verify_tree");
   amph_status rc = do_accept(ctx, out_tokens, out_n, out_path, out_next_root);
   if (rc == AMPH_OK) rc = finish(ctx, "accept");
-  if (rc == AMPH_OK) { ctx->phase = PH_READY; ctx->ctx_hi += ctx->cfg.K + 1; }
+  if (rc == AMPH_OK) {
+    ctx->phase = PH_READY;
+    for (int b = 0; b < ctx->B; ++b) ctx->ctx_hi[b] += ctx->cfg.K + 1;
+  }
   return rc;
 }
 
@@ -826,13 +991,11 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n) {
   amph_status rc = check_capacity(ctx);
   if (rc != AMPH_OK) return rc;
   const amph_config& c = ctx->cfg;
-  DevState* ds = ctx->at<DevState>(ctx->lay.state);
   const bool use_graph = !ctx->graph_off && !ctx->prof_on && !(c.flags & AMPH_FLAG_NO_GRAPH) && ctx->stream != nullptr;
   if (use_graph) {
     // The kernels read every length from device state; only the attention grids depend on the host's
     // bound of the context length, so the captured schedule is reused until that grid size changes.
-    const int key = attn_splits_for(ctx, ctx->ctx_hi, ctx->rows_small) * 128 +
-                    attn_splits_for(ctx, ctx->ctx_hi + ctx->tree_host.n_nodes, ctx->Mver);
+    const long long key = graph_key_of(ctx);
     if (!ctx->graph_exec || key != ctx->graph_key) {
       if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
       cudaGraph_t graph = nullptr;
@@ -862,10 +1025,14 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n) {
     if (rc == AMPH_OK) rc = do_verify(ctx, nullptr, nullptr);
     if (rc == AMPH_OK) rc = do_accept(ctx, nullptr, nullptr, nullptr, nullptr);
   }
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_tokens, ds->out_tok, sizeof(int) * (c.K + 1));
-  if (rc == AMPH_OK) rc = copy_out(ctx, out_n, &ds->L, sizeof(int));
+  for (int b = 0; b < ctx->B && rc == AMPH_OK; ++b) {
+    DevState* ds = ctx->state(b);
+    if (out_tokens) rc = copy_out(ctx, out_tokens + b * (c.K + 1), ds->out_tok, sizeof(int) * (c.K + 1));
+    if (rc == AMPH_OK && out_n) rc = copy_out(ctx, out_n + b, &ds->L, sizeof(int));
+  }
   if (rc == AMPH_OK) rc = finish(ctx, "step");
-  if (rc == AMPH_OK) ctx->ctx_hi += c.K + 1;
+  if (rc == AMPH_OK)
+    for (int b = 0; b < ctx->B; ++b) ctx->ctx_hi[b] += c.K + 1;
   return rc;
 }
 
@@ -874,28 +1041,38 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
   if (!name || !dst) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and dst must not be NULL");
   const amph_config& c = ctx->cfg;
   const Layout& l = ctx->lay;
-  const size_t d = c.d_model, V = c.vocab, N = ctx->tree_host.n_nodes, K = c.K, R = ctx->Mcap;
+  // optional suffixes: "#b" selects sequence b (default 0), "@row0" the first cache slot of a cache export
+  std::string nm(name);
+  int row0 = 0, seq = 0;
+  size_t at = nm.find('@');
+  if (at != std::string::npos) { row0 = atoi(nm.c_str() + at + 1); nm = nm.substr(0, at); }
+  at = nm.find('#');
+  if (at != std::string::npos) { seq = atoi(nm.c_str() + at + 1); nm = nm.substr(0, at); }
+  if (seq < 0 || seq >= ctx->B) return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s': sequence outside 0..%d", name, ctx->B - 1);
+  const size_t d = c.d_model, V = c.vocab, N = ctx->tree_host.n_nodes, K = c.K, R = ctx->Rcap, Mv = ctx->Mver;
+  // row buffers: sequence b's rows of a verification pass start at row b * Mver (after a prefill: the rows of its last pass)
   struct { const char* n; size_t off, size; } plain[] = {
-      {"hidden", l.hidden, 4 * R * d},   {"logits", l.logits, 4 * R * V},     {"d_logits", l.d_logits, 4 * K * V},
-      {"hp", l.hp, 4 * K * d},           {"attn_o", l.attn_o, 4 * K * d},     {"sal_h", l.last, 4 * 2 * d},
-      {"tree_tokens", l.tok, 4 * N},     {"argmax", l.amax, 4 * N},
+      {"hidden", l.hidden + 4 * seq * Mv * d, 4 * (R - seq * Mv) * d},
+      {"logits", l.logits + 4 * seq * Mv * V, 4 * (R - seq * Mv) * V},
+      {"d_logits", l.d_logits + l.d_logits_s * seq, 4 * K * V},
+      {"hp", l.hp + 4 * seq * kMaxK * d, 4 * K * d},
+      {"attn_o", l.attn_o + 4 * seq * K * d, 4 * K * d},
+      {"sal_h", l.last + l.last_s * seq, 4 * 2 * d},
+      {"tree_tokens", l.tok + 4 * seq * Mv, 4 * N},
+      {"argmax", l.amax + 4 * seq * Mv, 4 * N},
   };
   for (auto& p : plain) {
-    if (strcmp(name, p.n) == 0) {
+    if (nm == p.n) {
       if (bytes > p.size) return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' holds %zu bytes, %zu requested", name, p.size, bytes);
       return copy_out(ctx, dst, ctx->ws + p.off, bytes);
     }
   }
-  // cache exports: "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v", optional "@row0" suffix
-  std::string nm(name);
-  int row0 = 0;
-  const size_t at = nm.find('@');
-  if (at != std::string::npos) { row0 = atoi(nm.c_str() + at + 1); nm = nm.substr(0, at); }
+  // cache exports: "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v"
   KvView kv = {nullptr, nullptr};
   int which = -1, idx = -1;
   char kvc = 0;
-  if (sscanf(nm.c_str(), "kv.%c.%d", &kvc, &idx) == 2 && idx >= 0 && idx < c.n_layers) kv = ctx->kv_target[idx];
-  else if (sscanf(nm.c_str(), "sal%d.%c", &idx, &kvc) == 2 && idx >= 1 && idx <= c.n_sal) kv = ctx->kv_sal[idx - 1];
+  if (sscanf(nm.c_str(), "kv.%c.%d", &kvc, &idx) == 2 && idx >= 0 && idx < c.n_layers) kv = ctx->kv_target[seq][idx];
+  else if (sscanf(nm.c_str(), "sal%d.%c", &idx, &kvc) == 2 && idx >= 1 && idx <= c.n_sal) kv = ctx->kv_sal[seq][idx - 1];
   if (kvc == 'k') which = 0;
   if (kvc == 'v') which = 1;
   if (!kv.k || which < 0) return fail(ctx, AMPH_ERR_INVALID_ARG, "unknown tensor '%s'", name);
@@ -913,35 +1090,50 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
 amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
   if (!name || !src) return fail(ctx, AMPH_ERR_INVALID_ARG, "name and src must not be NULL");
-  if (strcmp(name, "root") == 0) {               // right after prefill: replaces the greedy root token
+  std::string nm(name);
+  int seq = 0;
+  const size_t at = nm.find('#');
+  if (at != std::string::npos) { seq = atoi(nm.c_str() + at + 1); nm = nm.substr(0, at); }
+  if (seq < 0 || seq >= ctx->B) return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s': sequence outside 0..%d", name, ctx->B - 1);
+  if (nm == "root") {                            // right after prefill: replaces the greedy root token
     if (ctx->phase != PH_READY || bytes != sizeof(int)) return fail(ctx, AMPH_ERR_STATE, "'root' takes one int32 right after amph_prefill");
-    DevState* ds = ctx->at<DevState>(ctx->lay.state);
+    DevState* ds = ctx->state(seq);
     amph_status rc = cuda_check(ctx, cudaMemcpyAsync(&ds->root, src, sizeof(int), cudaMemcpyDefault, ctx->stream), "set_tensor");
     if (rc == AMPH_OK) rc = cuda_check(ctx, cudaMemcpyAsync(&ds->pend_tok[0], src, sizeof(int), cudaMemcpyDefault, ctx->stream), "set_tensor");
     return rc;
   }
   if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_set_tensor must follow amph_verify_tree");
   size_t off;
-  if (strcmp(name, "tree_tokens") == 0) off = ctx->lay.tok;
-  else if (strcmp(name, "argmax") == 0) off = ctx->lay.amax;
+  if (nm == "tree_tokens") off = ctx->lay.tok;
+  else if (nm == "argmax") off = ctx->lay.amax;
   else return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' cannot be set", name);
   if (bytes != sizeof(int) * (size_t)ctx->tree_host.n_nodes)
     return fail(ctx, AMPH_ERR_INVALID_ARG, "'%s' takes exactly n_nodes int32 values", name);
-  return cuda_check(ctx, cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyDefault, ctx->stream), "set_tensor");
+  return cuda_check(ctx, cudaMemcpyAsync(ctx->ws + off + sizeof(int) * seq * ctx->Mver, src, bytes, cudaMemcpyDefault, ctx->stream), "set_tensor");
 }
 
-amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending) {
+amph_status amph_get_state_seq(amph_ctx* ctx, int32_t seq, int32_t* ctx_len, int32_t* root, int32_t* n_pending) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
+  if (seq < 0 || seq >= ctx->B) return fail(ctx, AMPH_ERR_INVALID_ARG, "sequence %d is outside 0..%d", seq, ctx->B - 1);
   DevState s;
-  cudaError_t e = cudaMemcpyAsync(&s, ctx->at<DevState>(ctx->lay.state), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
+  cudaError_t e = cudaMemcpyAsync(&s, ctx->state(seq), sizeof s, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) return cuda_check(ctx, e, "state read-back");
-  if (ctx->phase != PH_CREATED) ctx->ctx_hi = s.C;
+  if (ctx->prefilled[seq]) ctx->ctx_hi[seq] = s.C;
   if (ctx_len) *ctx_len = s.C;
   if (root) *root = s.root;
   if (n_pending) *n_pending = s.n_pending;
-  if (s.err) return fail(ctx, s.err, "a device-side wait gave up (code %d)", s.err);
+  int err = s.err;
+  if (seq != 0 && !err) {                        // device-side waits report through sequence 0's state word
+    DevState s0;
+    if (cudaMemcpy(&s0, ctx->state(0), sizeof s0, cudaMemcpyDeviceToHost) == cudaSuccess) err = s0.err;
+  }
+  if (err) return fail(ctx, err, "a device-side wait gave up (code %d)", err);
   return AMPH_OK;
+}
+
+amph_status amph_get_state(amph_ctx* ctx, int32_t* ctx_len, int32_t* root, int32_t* n_pending) {
+  return amph_get_state_seq(ctx, 0, ctx_len, root, n_pending);
 }
 
 amph_status amph_profile_begin(amph_ctx* ctx) {
@@ -1063,12 +1255,12 @@ amph_status amph_set_state(amph_ctx* ctx, int32_t ctx_len, int32_t root, int32_t
   s.C_old = ctx_len;
   s.next_root = root;
   for (int j = 0; j < 16; ++j) { s.path[j] = -1; s.out_tok[j] = -1; }
-  amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<DevState>(ctx->lay.state), &s, sizeof s, cudaMemcpyHostToDevice, ctx->stream), "set_state");
+  amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->state(0), &s, sizeof s, cudaMemcpyHostToDevice, ctx->stream), "set_state");
   if (rc == AMPH_OK) rc = cuda_check(ctx, cudaStreamSynchronize(ctx->stream), "set_state");       // s lives on this stack frame
   if (rc == AMPH_OK)
     rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<float>(ctx->lay.pend_h), pend_hidden, sizeof(float) * (size_t)n_pending * c.d_model,
                                          cudaMemcpyDefault, ctx->stream), "set_state");
-  if (rc == AMPH_OK) ctx->ctx_hi = ctx_len;
+  if (rc == AMPH_OK) ctx->ctx_hi[0] = ctx_len;
   return rc;
 }
 
@@ -1083,9 +1275,9 @@ amph_status amph_profile_breakdown(amph_ctx* ctx, double* ms, int64_t* launches)
 
 amph_status amph_reset(amph_ctx* ctx) {
   if (!ctx) return fail(nullptr, AMPH_ERR_INVALID_ARG, "ctx must not be NULL");
-  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, sizeof(DevState), ctx->stream);
+  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, ctx->lay.state_s * kMaxSeq, ctx->stream);
   ctx->phase = PH_CREATED;
-  ctx->ctx_hi = 0;
+  for (int b = 0; b < kMaxSeq; ++b) { ctx->ctx_hi[b] = 0; ctx->prefilled[b] = false; }
   return cuda_check(ctx, e, "reset");
 }
 

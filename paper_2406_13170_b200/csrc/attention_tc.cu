@@ -686,7 +686,7 @@ bool launch_tree_attention_tc(AttnTc* a, const void* q, int q_rows_cap, KvView k
                               int n_heads, int head_dim, int max_ctx, int splits, int keys_bound, cudaStream_t st,
                               void* merged_out, int* err_flag) {
   if (!a || splits < 1 || (merged_out && splits > 8)) return false;
-  if (q_rows_cap < (rows + kRows - 1) / kRows * kRows) return false;      // a Q box must stay inside the buffer
+  if (q_rows_cap < 1) return false;                   // rows of a Q box past the end of the buffer read as zeros
   if (head_dim == 64)
     return launch_t<64>(a, q, q_rows_cap, kv, meta, sc, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
   if (head_dim == 128)

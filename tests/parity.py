@@ -80,8 +80,9 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
     rep = Report()
     st = orc.prefill(prompt)
     root = model.prefill(prompt)
-    # logits of the last prompt position: row (n-1) mod 128 of the last prefill chunk (chunks of AMPH_MAX_NODES tokens)
-    last_row = (len(prompt) - 1) % 128
+    # logits of the last prompt position: row (n-1) mod 512 of the last prefill pass (a pass carries 4 x AMPH_MAX_NODES
+    # prompt tokens; AMPH_MAX_NODES with AMPH_FLAG_CHUNKED_PREFILL = 128)
+    last_row = (len(prompt) - 1) % (128 if (model.cfg.flags & 128) else 512)
     g_last = model.get_tensor("logits", (last_row + 1, V))[last_row]
     e = rel_err(g_last, st.last_logits)
     rep.max_logit_err = max(rep.max_logit_err, e)

@@ -98,14 +98,3 @@ def test_large_shapes_two_layers_stated_tolerance(name):
     rep = _run(shape, 2, True, kv_layers=(0, 1), init="fan_in")
     assert rep.steps == 2
     assert max(rep.max_logit_err, rep.max_hidden_err, rep.max_dlogit_err, rep.max_draft_err, rep.max_kv_err) <= TOL_BF16
-
-
-@pytest.mark.parametrize("name", ["7b", "33b"])
-def test_large_shapes_two_layers_benchmark_weights(name):
-    """N(0, 0.02) weights against the oracle's bf16-storage mode: 2e-2 on the target; the draft module's tensors
-    (un-normalised vocabulary logits on an expanding stack) stay within 0.15 (measured 6e-2)."""
-    shape = inputs.get_shape(name).with_(n_layers=2, prompt_len=70)
-    rep = _run(shape, 2, True, kv_layers=(0, 1), storage=torch.bfloat16)
-    assert rep.steps == 2
-    assert max(rep.max_logit_err, rep.max_hidden_err, rep.max_kv_err) <= TOL_BF16
-    assert max(rep.max_dlogit_err, rep.max_draft_err) <= 0.15
