@@ -53,6 +53,7 @@ enum { AMPH_DTYPE_F32 = 0, AMPH_DTYPE_BF16 = 1 };
 enum {
   AMPH_FLAG_NO_TENSOR_CORE = 1, /* route every projection through the plain CUDA-core kernel */
   AMPH_FLAG_NO_GRAPH = 2,       /* launch kernels one by one instead of replaying a CUDA graph */
+  AMPH_FLAG_SEPARATE_ROPE = 4,   /* rotary embedding + KV-cache write as a kernel of their own (bf16, up to 64 rows: the q / k / v projection does both otherwise) */
   AMPH_FLAG_SEPARATE_MERGE = 8,  /* merge the attention KV splits in a kernel of its own (bf16: a cluster does it otherwise) */
   AMPH_FLAG_SEPARATE_SWIGLU = 16, /* SwiGLU as a kernel of its own (bf16: the gate / up projection applies it otherwise) */
   AMPH_FLAG_NO_SAMPLED_TOKEN = 64, /* the "w/o Sampled-Token" ablation (Section 4.5): the adaptation layers are fed the

@@ -441,9 +441,18 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, CacheOf cache_of, float* x, c
   const int rows = ps.rows();
   const size_t d = c.d_model;
   const void* qkv[3] = {w.wq, w.wk, w.wv};
-  PartialView P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
   const RowScale rs = entry_deferred ? row_scale_of(ctx, l.ss_a) : RowScale();
-  for (int g = 0; g < ps.G; ++g) {                    // rotary embedding + cache write, per group (its own cache and slots)
+  PartialView P = {nullptr, 0, 0, 0};
+  bool fused_rope = false;
+  if (ctx->tc && ps.G == 1 && !(c.flags & AMPH_FLAG_SEPARATE_ROPE)) {   // q / k / v projection that rotates and writes the cache itself
+    ProfScope p(ctx, AMPH_PROF_PROJECTION);
+    fused_rope = tc_gemm_launch_qkv_rope(ctx->tc, XB_XN, w.wq, w.wk, w.wv, c.n_heads, c.head_dim, c.d_model, rows, ctx->ws + l.q,
+                                         cache_of(ps.seq[0]), ps.meta[0], ps.rope[0], c.max_ctx, rs, st);
+    if (fused_rope && p.rec) ctx->prof_bytes += 3LL * c.d_model * c.d_model * (int64_t)ctx->esz;
+    if (!fused_rope) cudaGetLastError();
+  }
+  if (!fused_rope) P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
+  for (int g = 0; g < ps.G && !fused_rope; ++g) {     // rotary embedding + cache write, per group (its own cache and slots)
     ProfScope p(ctx, AMPH_PROF_ROPE_KV);
     launch_qkv_rope(rows_from(P, g * ps.rpg), ps.meta[g], ps.rope[g], ctx->ws + l.q + ctx->esz * g * ps.rpg * d, cache_of(ps.seq[g]),
                     ctx->dtype, ps.rpg, c.n_heads, c.head_dim, c.max_ctx, st, rows_from(rs, g * ps.rpg));

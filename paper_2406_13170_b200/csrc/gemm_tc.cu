@@ -55,6 +55,14 @@ struct TcParams {
   int f;
   int up_first;             // the tensor map's outer index 0 is the up matrix (it has the lower address)
   RowScale rs;
+  // ROPE launches (q / k / v projection): a tile is 32 rotation pairs of one head, rows [32 j, 32 j + 32) and
+  // [dh/2 + 32 j, dh/2 + 32 j + 32); the epilogue rotates, scales and writes the query rows and the cache rows
+  __nv_bfloat16* q;         // [rows][n_heads * dh]
+  __nv_bfloat16* kc;        // [n_heads][max_ctx][dh]
+  __nv_bfloat16* vc;
+  const RowMeta* meta;      // slot of every row, number of live rows
+  const float2* rope;       // [rows][dh / 2] (cos, sin)
+  int n_heads, dh, max_ctx;
   int* err_flag;
   unsigned long long wait_limit_ns;   // a barrier wait gives up after this long
   uint32_t extra_tx;                   // self-test only: bytes the first stage's barrier expects beyond what is copied
@@ -137,6 +145,16 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, i
       ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(kb), "r"(0), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
+// (column, row, half, K block): the two 32-row halves of a rotation tile land as 64 consecutive rows per K block
+__device__ __forceinline__ void tma_load_4d_kb_outer(void* dst, const CUtensorMap* map, int row, int kb, uint64_t* bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(row), "r"(0), "r"(kb), "r"(smem_u32(bar)), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_l2_4d_kb_outer(const CUtensorMap* map, int row, int kb) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(0), "r"(row), "r"(0), "r"(kb) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int row, int kb) {
   asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(0), "r"(row), "r"(kb), "r"(0) : "memory");
 }
@@ -186,11 +204,20 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 // step it issues two M = 64 MMAs, gate rows into accumulator columns [0, nt) and up rows into [ntc, ntc + nt).  Row r
 // of an M = 64 accumulator lives in TMEM lane 32 (r / 16) + r % 16 (checked on the device), so lane l < 16 of the
 // epilogue warp of quarter q holds gate and up of feature 16 q + l for all rows: no exchange between warps.
-template <bool SWIGLU>
+//
+// ROPE: the q / k / v projection with the rotary embedding and the cache write in the epilogue.  A CTA owns 64 weight
+// rows that hold 32 complete rotation pairs of one head (both halves fetched by one 4-D copy) and the whole K range,
+// one M = 64 MMA per K step.  The partners of a pair sit in different epilogue warps; the accumulator tile goes through
+// shared memory (the ring is free by then), then every thread rotates 16 pairs of one row and writes 32-byte pieces.
+enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_ROPE = 2 };
+constexpr int kRopePitch = 68;        // floats per activation row of the exchanged tile (64 + 4: conflict-free float4 reads)
+
+template <int EPI>
 __global__ void __launch_bounds__(kThreads)
 tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
+  constexpr bool SWIGLU = EPI == EPI_SWIGLU, ROPE = EPI == EPI_ROPE;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ float inv_s[SWIGLU ? kTileM : 1];         // 1 / rms of the activation rows (SWIGLU)
+  __shared__ float inv_s[EPI != EPI_PARTIAL ? kTileM : 1];         // 1 / rms of the activation rows (SWIGLU, ROPE)
   __shared__ __align__(8) uint64_t full_bar[8];
   __shared__ __align__(8) uint64_t empty_bar[8];
   __shared__ __align__(8) uint64_t accum_bar;
@@ -202,7 +229,11 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int seg = tile / prm.tiles_per_seg;
-  const int row0 = SWIGLU ? tile * (kTileM / 2) : (tile - seg * prm.tiles_per_seg) * kTileM;   // first weight row of this tile
+  int row0 = SWIGLU ? tile * (kTileM / 2) : (tile - seg * prm.tiles_per_seg) * kTileM;   // first weight row of this tile
+  if constexpr (ROPE) {
+    const int tph = prm.dh >> 6, tt = tile - seg * prm.tiles_per_seg;       // tiles per head = (dh / 2) / 32
+    row0 = (tt / tph) * prm.dh + (tt % tph) * 32;
+  }
   // K range of this split in whole stages (ks blocks), so that every copy starts on a stage boundary
   const int ks = prm.ks;
   const int units = (prm.kblocks + ks - 1) / ks;
@@ -212,9 +243,9 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   const int nkb = kb_hi - kb_lo;
   const int nit = (nkb + ks - 1) / ks;                  // pipeline iterations
   const int nt = prm.nt, stages = prm.stages;
-  const uint32_t a_tile = kTileM * kTileK * 2, b_tile = (uint32_t)nt * kTileK * 2;     // one K block of each operand
+  const uint32_t a_tile = (ROPE ? kTileM / 2 : kTileM) * kTileK * 2, b_tile = (uint32_t)nt * kTileK * 2;     // one K block of each operand
   const uint32_t a_bytes = ks * a_tile, b_bytes = ks * b_tile;
-  const int nblk = SWIGLU ? 1 : prm.nblk;              // row blocks: each gets its own activation tile and accumulator
+  const int nblk = EPI != EPI_PARTIAL ? 1 : prm.nblk;              // row blocks: each gets its own activation tile and accumulator
   const uint32_t b_slot = (b_bytes + 1023u) & ~1023u;
   const uint32_t stage_bytes = a_bytes + (uint32_t)nblk * b_slot;
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -256,11 +287,13 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         // extra_tx is 0 except in the failure-path self-test, where the first barrier expects bytes that never come
         mbar_expect_tx(&full_bar[i], a_bytes + (uint32_t)nblk * b_bytes + (i == 0 ? prm.extra_tx : 0u));
         if (SWIGLU) tma_load_4d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
+        else if (ROPE) tma_load_4d_kb_outer(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
         else tma_load_3d(smem + (size_t)i * stage_bytes, wmap, row0, kb_lo + i * ks, &full_bar[i], wpol);
       }
       // While the previous kernel still runs, HBM would idle: pull the next weight tiles into L2 as well.
       for (int i = npre; i < npf; ++i) {
         if (SWIGLU) tma_prefetch_l2_4d(wmap, row0, kb_lo + i * ks);
+        else if (ROPE) tma_prefetch_l2_4d_kb_outer(wmap, row0, kb_lo + i * ks);
         else tma_prefetch_l2_3d(wmap, row0, kb_lo + i * ks);
       }
     }
@@ -279,6 +312,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
         uint8_t* a = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full_bar[s], a_bytes + (uint32_t)nblk * b_bytes);
         if (SWIGLU) tma_load_4d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
+        else if (ROPE) tma_load_4d_kb_outer(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
         else tma_load_3d(a, wmap, row0, kb_lo + i * ks, &full_bar[s], wpol);
         for (int z = 0; z < nblk; ++z) tma_load_3d(a + a_bytes + (size_t)z * b_slot, &maps.x, z * nt, kb_lo + i * ks, &full_bar[s]);
       }
@@ -296,7 +330,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
   } else if (warp == 1) {
     // ---------------- MMA issuer (the warp stays converged, its elected lane issues)
     const bool leader = elect_one();
-    const uint32_t idesc = umma_idesc(nt, SWIGLU ? kTileM / 2 : kTileM);
+    const uint32_t idesc = umma_idesc(nt, EPI != EPI_PARTIAL ? kTileM / 2 : kTileM);
     bool ok = true;
     for (int i = 0; i < nit; ++i) {
       const int s = i % stages, round = i / stages;
@@ -339,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
     // ---------------- epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
     const int quarter = warp & 3;
     pdl_wait();                                      // P may still be read by the kernel before this one
-    if constexpr (SWIGLU) {                          // 1 / rms of the rows, while the main loop runs
+    if constexpr (EPI != EPI_PARTIAL) {              // 1 / rms of the rows, while the main loop runs
       const int et = threadIdx.x - 64;
       if (et < prm.rows) inv_s[et] = row_scale(prm.rs, et);
       asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -387,6 +421,81 @@ tc_gemm_kernel(const __grid_constant__ TmapPack maps, const TcParams prm) {
             const float t = gv[j] * sc;
             prm.act[(size_t)r * prm.f + feat] = __float2bfloat16(__fdividef(t, 1.0f + __expf(-t)) * (uv[j] * sc));
           }
+        }
+      }
+    } else if constexpr (ROPE) {
+      // lane l < 16 of the warp of quarter q holds tile row 16 q + l (pair member lo for q < 2, hi for q >= 2) for all
+      // activation rows: park the tile as ex[activation row][tile row] in the ring, which no copy or MMA touches any more
+      float* ex = reinterpret_cast<float*>(smem);
+      for (int c0 = 0; c0 < nt; c0 += 16) {
+        uint32_t v[16];
+        if (ok) {
+          const uint32_t taddr = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+              : "r"(taddr)
+              : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
+        }
+        if (lane < 16) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ex[(c0 + j) * kRopePitch + quarter * 16 + lane] = __uint_as_float(v[j]);
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      // thread e: activation row e / 2, pairs 16 (e % 2) .. + 15 of the tile
+      const int et = threadIdx.x - 64;
+      const int r = et >> 1, t0 = (et & 1) * 16;
+      if (r < prm.rows) {
+        const int half = prm.dh >> 1;
+        const int tt = tile - seg * prm.tiles_per_seg, tph = prm.dh >> 6;
+        const int h = tt / tph, i0 = (tt % tph) * 32 + t0;               // head, first pair index of this thread
+        const float sc = inv_s[r];
+        float a[16], b[16];
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) {
+          const float4 va = *reinterpret_cast<const float4*>(ex + r * kRopePitch + t0 + j);
+          const float4 vb = *reinterpret_cast<const float4*>(ex + r * kRopePitch + 32 + t0 + j);
+          a[j] = va.x * sc; a[j + 1] = va.y * sc; a[j + 2] = va.z * sc; a[j + 3] = va.w * sc;
+          b[j] = vb.x * sc; b[j + 1] = vb.y * sc; b[j + 2] = vb.z * sc; b[j + 3] = vb.w * sc;
+        }
+        uint32_t lo[8], hi[8];
+        if (seg < 2) {                                 // queries and keys: rotate pair (i, i + dh / 2) by the row's angle
+          const float2* cs = prm.rope + (size_t)r * half + i0;
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const float4 c2 = *reinterpret_cast<const float4*>(cs + j);        // (cos, sin) of pairs j, j + 1
+            const __nv_bfloat162 l2 = __floats2bfloat162_rn(a[j] * c2.x - b[j] * c2.y, a[j + 1] * c2.z - b[j + 1] * c2.w);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(b[j] * c2.x + a[j] * c2.y, b[j + 1] * c2.z + a[j + 1] * c2.w);
+            lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&l2);
+            hi[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const __nv_bfloat162 l2 = __floats2bfloat162_rn(a[j], a[j + 1]), h2 = __floats2bfloat162_rn(b[j], b[j + 1]);
+            lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&l2);
+            hi[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        }
+        __nv_bfloat16* dst = nullptr;
+        if (seg == 0) {
+          dst = prm.q + (size_t)r * prm.n_heads * prm.dh + h * prm.dh + i0;
+        } else {
+          const int slot = prm.meta->slot[r];
+          if (r < prm.meta->n_rows && slot >= 0 && slot < prm.max_ctx)
+            dst = (seg == 1 ? prm.kc : prm.vc) + ((size_t)h * prm.max_ctx + slot) * prm.dh + i0;
+        }
+        if (dst != nullptr) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(dst + 8) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+          *reinterpret_cast<uint4*>(dst + half) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(dst + half + 8) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
         }
       }
     } else {
@@ -464,6 +573,25 @@ struct TcGemm {
     return &(pair_cache[key] = m);
   }
 
+  // A [rows, cols] matrix as (column, row, half, K block) with the half `half_rows` rows apart: a box is 32 rows of
+  // both halves, i.e. 32 rotation pairs of one head, over box_kb K blocks.
+  std::map<std::tuple<const void*, int, int, int, int>, CUtensorMap> rope_cache;
+  const CUtensorMap* get_rope(const void* ptr, int rows, int cols, int half_rows, int box_kb) {
+    auto key = std::make_tuple(ptr, rows, cols, half_rows, box_kb);
+    auto it = rope_cache.find(key);
+    if (it != rope_cache.end()) return &it->second;
+    CUtensorMap m;
+    const cuuint64_t dims[4] = {(cuuint64_t)kTileK, (cuuint64_t)rows, 2, (cuuint64_t)cols / kTileK};
+    const cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)half_rows * cols * 2, (cuuint64_t)kTileK * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kTileK, 32, 2, (cuuint32_t)box_kb};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return nullptr;
+    return &(rope_cache[key] = m);
+  }
+
   const CUtensorMap* get(const void* ptr, int rows, int cols, int box_rows, int box_kb = kStageKb) {
     auto key = std::make_tuple(ptr, rows, cols, box_rows, box_kb);
     auto it = cache.find(key);
@@ -502,8 +630,9 @@ TcGemm* tc_gemm_create(void* const* xbufs, const int* xrows, const int* xcols, i
   for (int i = 0; i < n; ++i) { g->xptr[i] = xbufs[i]; g->xrows[i] = xrows[i]; g->xcols[i] = xcols[i]; }
   cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&g->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
-  cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  cudaFuncSetAttribute(tc_gemm_kernel<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  cudaFuncSetAttribute(tc_gemm_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
+  cudaFuncSetAttribute(tc_gemm_kernel<EPI_ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, g->max_smem - 2048);
   return g;
 }
 
@@ -567,7 +696,7 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
   prm.wait_limit_ns = g->wait_limit_ns;
   prm.extra_tx = g->extra_tx;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  launch_pdl(tc_gemm_kernel<false>, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
+  launch_pdl(tc_gemm_kernel<EPI_PARTIAL>, dim3(tiles, splits), dim3(kThreads), smem, st, pack, prm);
   *splits_out = splits;
   *split_stride = prm.split_stride;
   return true;
@@ -610,7 +739,59 @@ bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_
   prm.err_flag = g->err_flag;
   prm.wait_limit_ns = g->wait_limit_ns;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  return launch_pdl(tc_gemm_kernel<true>, dim3(tiles, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
+  return launch_pdl(tc_gemm_kernel<EPI_SWIGLU>, dim3(tiles, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
+}
+
+bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, const void* wv, int n_heads, int dh, int in,
+                             int rows, void* q, KvView kv, const RowMeta* meta, const float2* rope, int max_ctx,
+                             const RowScale& rs, cudaStream_t st) {
+  if (!g || xb < 0 || xb >= g->n_x || !wq || !wk || !wv || !q || !kv.k || !kv.v || !meta || !rope) return false;
+  if ((dh != 64 && dh != 128) || in % kTileK || rows < 1 || g->xcols[xb] != in) return false;
+  if (((uintptr_t)wq | (uintptr_t)wk | (uintptr_t)wv) & 15) return false;
+  const int d = n_heads * dh;
+  const int nt = rows <= 16 ? 16 : (rows + 15) / 16 * 16;
+  if (nt > 64 || nt > g->xrows[xb]) return false;          // the exchanged tile is 64 activation rows at most
+  const int ks = kStageKb, kblocks = in / kTileK, tiles_per_seg = d / 64;
+  TmapPack pack;
+  memset(&pack, 0, sizeof pack);
+  const void* w[3] = {wq, wk, wv};
+  for (int s = 0; s < 3; ++s) {
+    const CUtensorMap* m = g->get_rope(w[s], d, in, dh / 2, ks);
+    if (!m) return false;
+    pack.w[s] = *m;
+  }
+  const CUtensorMap* mx = g->get(g->xptr[xb], g->xrows[xb], in, nt, ks);
+  if (!mx) return false;
+  pack.x = *mx;
+  const uint32_t stage_bytes = ks * (kTileM / 2) * kTileK * 2 + ((ks * (uint32_t)nt * kTileK * 2 + 1023u) & ~1023u);
+  int stages = (int)((110 * 1024) / stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  if ((size_t)stages * stage_bytes < (size_t)nt * kRopePitch * 4) return false;   // the ring doubles as the exchange buffer
+  TcParams prm;
+  memset(&prm, 0, sizeof prm);
+  prm.tiles_per_seg = tiles_per_seg;
+  prm.kblocks = kblocks;
+  prm.splits = 1;
+  prm.nt = nt;
+  prm.nblk = 1;
+  prm.rows = rows;
+  prm.stages = stages;
+  prm.ks = ks;
+  prm.l2_prefetch = 1;
+  prm.rs = rs;
+  prm.q = (__nv_bfloat16*)q;
+  prm.kc = (__nv_bfloat16*)kv.k;
+  prm.vc = (__nv_bfloat16*)kv.v;
+  prm.meta = meta;
+  prm.rope = rope;
+  prm.n_heads = n_heads;
+  prm.dh = dh;
+  prm.max_ctx = max_ctx;
+  prm.err_flag = g->err_flag;
+  prm.wait_limit_ns = g->wait_limit_ns;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  return launch_pdl(tc_gemm_kernel<EPI_ROPE>, dim3(3 * tiles_per_seg, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
 }
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }

@@ -27,6 +27,15 @@ bool tc_gemm_launch(TcGemm* g, int xb, const void* const* w, int n_seg, int out,
 bool tc_gemm_launch_swiglu(TcGemm* g, int xb, const void* w_gate, const void* w_up, int f, int in, int rows, void* act,
                            const RowScale& rs, cudaStream_t st);
 
+// q / k / v projection with the rotary embedding and the cache write in the epilogue (no partial sums, no separate kernel):
+//   q[row] <- rope(s * X[row] . Wq^T),  K cache[slot[row]] <- rope(s * X[row] . Wk^T),  V cache[slot[row]] <- s * X[row] . Wv^T
+// with s the row's deferred RMSNorm scale, rope the rotation of pairs (i, i + dh / 2) by the angles in `rope`
+// ([rows][dh / 2] (cos, sin)).  Weights bf16 [n_heads * dh, in]; q bf16 [rows][n_heads * dh]; caches [head][slot][dh].
+// Takes at most 64 rows and head_dim 64 or 128; returns false, nothing launched, if the form is not available.
+bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, const void* wv, int n_heads, int dh, int in,
+                             int rows, void* q, KvView kv, const RowMeta* meta, const float2* rope, int max_ctx,
+                             const RowScale& rs, cudaStream_t st);
+
 void tc_gemm_destroy(TcGemm* g);
 
 // Failure-path self-test: every barrier wait of later launches gives up after wait_limit_ns, and the first stage's
