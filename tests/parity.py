@@ -197,3 +197,109 @@ def run_parity(model, orc: ao.Oracle, shape, topo, prompt: List[int], steps: int
             rep.max_kv_err = max(rep.max_kv_err, e)
             assert e <= tol_draft, f"stage {s+1} {which} cache off by {e}"
     return rep
+
+
+def run_parity_batch(model, borc, shape, topo, prompts: List[List[int]], steps: int, tol: float, tie_tol: float,
+                     futures: Optional[List[List[int]]] = None) -> List[Report]:
+    """The same protocol for max_batch sequences decoded side by side (Section 4.4): `borc` is the batched oracle
+    (oracle.amphista_batch_oracle.BatchOracle), prompts one list per sequence (lengths may differ).  With `futures`
+    (each sequence's true greedy continuation) a path of a different depth is planted per sequence and step, so that
+    the sequences accept different numbers of tokens and their lengths drift apart.  One Report per sequence."""
+    dev = model.device
+    t = ao.tree_tables(topo.parent, topo.depth, topo.rank)
+    N, K, d, V, B = t.n_nodes, shape.K, shape.d_model, shape.vocab, len(prompts)
+    reps = [Report() for _ in range(B)]
+    bs = borc.prefill(prompts)
+    for b in range(B):
+        root = model.prefill(prompts[b], seq=b)
+        if root != bs.root[b]:
+            top2 = torch.topk(bs.last_logits[b].to(torch.float64), 2).values
+            assert float(top2[0] - top2[1]) <= 2.0 * tol * max(1.0, float(bs.last_logits[b].abs().max())), \
+                f"sequence {b}: prefill root {root} vs oracle {bs.root[b]}"
+            reps[b].argmax_near_ties += 1
+            model.set_tensor(f"root#{b}", torch.tensor([bs.root[b]], dtype=torch.int32, device=dev))
+    done = [0] * B
+    g_ids = torch.zeros(B, K, 16, dtype=torch.int32, device=dev)
+    g_vals = torch.zeros(B, K, 16, dtype=torch.float32, device=dev)
+    g_amax = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    g_tok = torch.zeros(B, K + 1, dtype=torch.int32, device=dev)
+    g_path = torch.zeros(B, K + 1, dtype=torch.int32, device=dev)
+    g_n = torch.zeros(B, dtype=torch.int32, device=dev)
+    g_next = torch.zeros(B, dtype=torch.int32, device=dev)
+    for i in range(steps):
+        C0 = list(bs.C)
+        for b in range(B):
+            assert model.get_state(b)[0] == C0[b]
+        ovs = None
+        if futures is not None:
+            ovs = []
+            for b in range(B):
+                leaf = t.leaves[(i + 2 * b) % len(t.leaves)]
+                ovs.append(plant(t, futures[b][done[b] + 1: done[b] + 1 + t.depth[leaf]], leaf) if (i + b) % 3 else None)
+        taps = [dict() for _ in range(B)]
+        emitted = borc.step(bs, t, ovs, taps)
+        model.draft(g_ids, g_vals)
+        torch.cuda.synchronize(dev)
+        for b in range(B):
+            tp, rep = taps[b], reps[b]
+            g_dl = model.get_tensor(f"d_logits#{b}", (K, V))
+            e_dl = rel_err(g_dl, tp["d_logits"])
+            e_hp = rel_err(model.get_tensor(f"hp#{b}", (K, d)), tp["Hp"])
+            e_ao = rel_err(model.get_tensor(f"attn_o#{b}", (K, d)), tp["attn_o"])
+            sal_h = model.get_tensor(f"sal_h#{b}", (2, d))
+            e_h = max(rel_err(sal_h[0], tp["h1"]), rel_err(sal_h[1], tp["h2"]))
+            rep.max_dlogit_err = max(rep.max_dlogit_err, e_dl)
+            rep.max_draft_err = max(rep.max_draft_err, e_hp, e_ao, e_h)
+            assert max(e_dl, e_hp, e_ao, e_h) <= tol, f"step {i} sequence {b}: draft tensors off by {(e_dl, e_hp, e_ao, e_h)}"
+            scale = max(1.0, float(tp["d_logits"].abs().max()))
+            e_abs = float((g_dl.to(torch.float64).cpu() - tp["d_logits"].to(torch.float64)).abs().max())
+            compare_topk(shape, g_ids[b], g_vals[b], tp["d_logits"], max(tie_tol * scale, 2.0 * e_abs), rep)
+            g_tt = model.get_tensor(f"tree_tokens#{b}", (N,), torch.int32).tolist()
+            assert g_tt == ao.Oracle.tree_tokens(int(tp["toks"][0]), g_ids[b].tolist(), t), f"step {i} sequence {b}: tree tokens"
+        model.verify_tree(torch.tensor([tp["toks"] for tp in taps], dtype=torch.int32, device=dev), g_amax)
+        torch.cuda.synchronize(dev)
+        for b in range(B):
+            tp, rep = taps[b], reps[b]
+            g_logits = model.get_tensor(f"logits#{b}", (N, V))
+            g_hidden = model.get_tensor(f"hidden#{b}", (N, d))
+            le, he = rel_err(g_logits, tp["logits"]), rel_err(g_hidden, tp["hid"])
+            rep.max_logit_err, rep.max_hidden_err = max(rep.max_logit_err, le), max(rep.max_hidden_err, he)
+            assert max(le, he) <= tol, f"step {i} sequence {b}: logits / hidden off by {(le, he)}"
+            lscale = max(1.0, float(tp["logits"].abs().max()))
+            top2 = torch.topk(tp["logits"].to(torch.float64), 2, dim=1).values
+            e_log = float((g_logits.to(torch.float64).cpu() - tp["logits"].to(torch.float64)).abs().max())
+            safe = (top2[:, 0] - top2[:, 1]) > max(2.0 * e_log, 1e-6 * lscale)
+            ga = g_amax[b].tolist()
+            for n in range(N):
+                if bool(safe[n]):
+                    assert ga[n] == tp["amax"][n], f"step {i} sequence {b} node {n}: argmax {ga[n]} vs {tp['amax'][n]}"
+                else:
+                    rep.argmax_near_ties += 1
+            if not bool(safe.all()):
+                rep.gated_steps += 1
+                model.set_tensor(f"argmax#{b}", torch.tensor(tp["amax"], dtype=torch.int32, device=dev))
+        model.accept(g_tok, g_n, g_path, g_next)
+        torch.cuda.synchronize(dev)
+        for b in range(B):
+            tp, rep = taps[b], reps[b]
+            L = int(g_n[b])
+            assert L == tp["L"], f"step {i} sequence {b}: accepted {L} vs oracle {tp['L']}"
+            assert g_path[b, :L].tolist() == tp["path"] and g_tok[b, :L].tolist() == emitted[b]
+            assert int(g_next[b]) == tp["next_root"]
+            assert model.get_state(b) == (bs.C[b], bs.root[b], L)
+            for which, cache in (("k", bs.K[0]), ("v", bs.V[0])):       # compacted rows of the first layer, this sequence's cache
+                rows = model.get_tensor(f"kv.{which}.0#{b}@{C0[b]}", (L, d))
+                e = rel_err(rows, cache[b, C0[b]:C0[b] + L])
+                rep.max_kv_err = max(rep.max_kv_err, e)
+                assert e <= tol, f"step {i} sequence {b}: {which} cache rows off by {e}"
+            done[b] += L
+            rep.accepted.append(L)
+            rep.steps += 1
+    for b in range(B):                                                  # adaptation-layer caches, per sequence
+        for s in range(shape.n_sal):
+            n_rows = bs.C[b] - len(bs.pending[b])
+            rows = model.get_tensor(f"sal{s+1}.k#{b}", (n_rows, d))
+            e = rel_err(rows, bs.sal_K[s][b, :n_rows])
+            reps[b].max_kv_err = max(reps[b].max_kv_err, e)
+            assert e <= tol, f"sequence {b}: stage {s+1} cache off by {e}"
+    return reps
