@@ -201,7 +201,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
   constexpr uint32_t kStage = 2 * NB * kKvBlock;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t q_full, p_ready, o_full;
-  __shared__ __align__(8) uint64_t k_full[4], v_full[4], kv_empty[4], s_full;
+  __shared__ __align__(8) uint64_t k_full[4], v_full[4], k_empty[4], v_empty[4], s_full;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
@@ -218,7 +218,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
     mbar_init(&q_full, 1);
     mbar_init(&p_ready, 128);
     mbar_init(&o_full, 1);
-    for (int s = 0; s < 4; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    for (int s = 0; s < 4; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_empty[s], 1); }
     mbar_init(&s_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -261,6 +261,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.v) : "memory");
     }
     int issued = 0;
+    bool k_only = false;                               // gave up between the key and the value copies of chunk `issued`
     // committed context: nothing the previous kernel writes
     if (leader) {
       while (issued < n_chunks && issued < stages && s_lo + (issued + 1) * kChunk <= base) {
@@ -281,12 +282,18 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
     }
     for (int c = issued; c < n_chunks; ++c) {
       const int st = c % stages, round = c / stages;
-      if (round > 0 && !__all_sync(0xffffffffu, mbar_wait(&kv_empty[st], (round & 1) ^ 1, &abort_flag))) break;
+      // the key half of a stage is free once the scores that read it are complete, the value half once P V is: the next
+      // keys arrive while this chunk's softmax and P V run, the next values while the next scores and softmax run
+      uint8_t* kdst = St + (size_t)st * kStage;
+      if (round > 0 && !__all_sync(0xffffffffu, mbar_wait(&k_empty[st], (round & 1) ^ 1, &abort_flag))) break;
       if (leader) {
-        uint8_t* kdst = St + (size_t)st * kStage;
         mbar_expect_tx(&k_full[st], NB * kKvBlock);
-        mbar_expect_tx(&v_full[st], NB * kKvBlock);
         for (int j = 0; j < NB; ++j) tma_load_3d(kdst + j * kKvBlock, &maps.k, 64 * j, s_lo + c * kChunk, h, &k_full[st]);
+      }
+      __syncwarp();
+      if (round > 0 && !__all_sync(0xffffffffu, mbar_wait(&v_empty[st], (round & 1) ^ 1, &abort_flag))) { k_only = true; break; }
+      if (leader) {
+        mbar_expect_tx(&v_full[st], NB * kKvBlock);
         for (int j = 0; j < NB; ++j) tma_load_3d(kdst + (NB + j) * kKvBlock, &maps.v, 64 * j, s_lo + c * kChunk, h, &v_full[st]);
       }
       __syncwarp();
@@ -299,6 +306,8 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
         const int st = c % stages, round = c / stages;
         while (!(mbar_try(&k_full[st], round & 1) && mbar_try(&v_full[st], round & 1)) && now_ns() - t0 < kWaitLimitNs) {}
       }
+      if (k_only && issued < n_chunks)
+        while (!mbar_try(&k_full[issued % stages], (issued / stages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
       if (n_chunks > 0) while (!mbar_try(&q_full, 0) && now_ns() - t0 < kWaitLimitNs) {}
     }
   } else if (warp == 1) {
@@ -317,6 +326,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
           umma_f16(d, umma_desc(q_addr + j * kQBlock) + (uint64_t)(2 * k), umma_desc(k_addr + j * kKvBlock) + (uint64_t)(2 * k),
                    idesc_s, (j | k) ? 1u : 0u);
       umma_commit(&s_full);
+      umma_commit(&k_empty[c % stages]);
     };
     bool ok = n_chunks > 0;
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&q_full, 0, &abort_flag));
@@ -344,7 +354,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
             umma_f16(tmem + kChunk + 64 * j, adesc, umma_desc_mn(v_addr + j * kKvBlock + (uint32_t)k * 2048), idesc_o, k ? 1u : 0u);
         }
         umma_commit(&o_full);
-        umma_commit(&kv_empty[st]);
+        umma_commit(&v_empty[st]);
       }
       __syncwarp();
       if (c + 1 < n_chunks) {                          // scores of the next chunk (the softmax has read this chunk's)
