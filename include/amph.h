@@ -95,6 +95,10 @@ typedef struct {
   int32_t lm_rank;        /* 0: each drafting head owns a [vocab, d] matrix (Eq. 6); r > 0: it owns two
                            * low-rank factors a [r, d] and b [vocab, r], logits = b (a x) (Appendix A.2.4);
                            * r a multiple of 8, r <= d_model                                  */
+  float temperature;      /* 0: greedy decoding (Table 1).  T > 0: random sampling (Table 2): the target draws every
+                           * token from softmax(logits / T), and a drafted token is accepted by the rejection-sampling
+                           * test of Section 2 for a point-mass proposal (see amph_accept)                        */
+  uint32_t seed_lo, seed_hi; /* key of the counter-based generator (Philox4x32-10) that supplies the uniforms at T > 0 */
 } amph_config;
 
 /* Draft-tree topology (Appendix A.1): node 0 is the root (the token the target chose last);
@@ -181,6 +185,15 @@ amph_status amph_verify_tree(amph_ctx* ctx, const int32_t* tree_tokens, int32_t*
 /* Greedy acceptance (Section 2): the deepest root path on which every drafted token equals the
  * target's greedy choice at its parent; compacts the accepted nodes' key / value rows to slots
  * ctx_len .. ctx_len + n - 1, advances ctx_len by n, and queues the accepted rows for the next draft.
+ * With temperature T > 0 the "choice" after node n is drawn instead (amph_verify_tree computes it right after the
+ * logits): with p = softmax(logits_n / T) and the node's uniform u_n, walk the vocabulary in the order (tokens of n's
+ * children in node order, then every other id ascending) and take the first token whose cumulative probability
+ * exceeds u_n.  Child i is thus accepted with probability p(x_i) / (1 - p(x_1) - .. - p(x_{i-1})) given that its elder
+ * siblings were rejected, and a node whose children are all rejected hands on a token drawn from p with the
+ * children's tokens removed: rejection sampling with point-mass proposals, which leaves the emitted tokens
+ * distributed exactly as sampling from the target.  u_n = 2^-24 * (top 24 bits of word 0 of Philox4x32-10 with counter
+ * (n, step, sequence, 0) and key (seed_lo, seed_hi)), step = acceptances the sequence has seen; the token after the
+ * prompt uses counter (0, 0, sequence, 1).
  * out_tokens [K+1], out_n [1], out_path [K+1] (node ids), out_next_root [1]: host or device int32,
  * each may be NULL. */
 amph_status amph_accept(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n, int32_t* out_path,
@@ -196,7 +209,8 @@ amph_status amph_step(amph_ctx* ctx, int32_t* out_tokens, int32_t* out_n);
  *   n_nodes after amph_verify_tree; after amph_prefill the rows of its last pass: a pass carries 4 * AMPH_MAX_NODES
  *   prompt tokens, so prompt token j is row j mod 512; AMPH_MAX_NODES with AMPH_FLAG_CHUNKED_PREFILL);
  *   "d_logits" f32 [K,V]; "hp" f32 [K,d] (Eq. 4); "attn_o" f32 [K,d] (Eq. 5);
- *   "sal_h" f32 [2,d] (Eq. 1: h^1_t, h^2_t of the last row); "tree_tokens", "argmax" i32 [n_nodes];
+ *   "sal_h" f32 [2,d] (Eq. 1: h^1_t, h^2_t of the last row); "tree_tokens", "argmax" i32 [n_nodes] (at T > 0
+ *   "argmax" holds the sampled choices); "uniforms" f32 [n_nodes] (the uniforms of the last verification, T > 0);
  *   "kv.k.{i}", "kv.v.{i}", "sal{s}.k", "sal{s}.v": f32 [rows, d] for cache slots 0..rows-1,
  *   rows = bytes / (4 d), converted from the cache's storage type.
  * bytes must not exceed the tensor's size. */
@@ -204,7 +218,8 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
 
 /* Test hook: overwrites "tree_tokens" or "argmax" (i32 [n_nodes], host or device source) with a
  * stream-ordered copy, e.g. to run amph_accept on a chosen verification outcome.  Allowed after
- * amph_verify_tree only.  "root" (i32 [1]) replaces the root token; allowed right after amph_prefill only.
+ * amph_verify_tree only.  "logits" (f32 [n_nodes, vocab], T > 0 only) replaces the verified rows' logits and draws
+ * the choices again from them with the same uniforms.  "root" (i32 [1]) replaces the root token; allowed right after amph_prefill only.
  * "#b" selects the sequence as for amph_get_tensor. */
 amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, size_t bytes);
 

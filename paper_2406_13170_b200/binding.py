@@ -35,7 +35,7 @@ class amph_config(C.Structure):
                 ("weight_dtype", C.c_int32), ("kv_dtype", C.c_int32), ("max_ctx", C.c_int32),
                 ("max_batch", C.c_int32), ("K", C.c_int32), ("n_sal", C.c_int32),
                 ("aeb_layers", C.c_int32), ("topk", C.c_int32 * AMPH_MAX_HEADS_K), ("flags", C.c_int32),
-                ("lm_rank", C.c_int32)]
+                ("lm_rank", C.c_int32), ("temperature", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
 class amph_tree(C.Structure):
@@ -108,7 +108,8 @@ def lib() -> C.CDLL:
     return _lib
 
 
-def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0, max_batch: int = 1) -> amph_config:
+def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0, max_batch: int = 1, temperature: float = 0.0,
+                seed: int = 0) -> amph_config:
     """amph_config from an object with the fields of inputs.configs.ModelShape."""
     c = amph_config()
     c.n_layers, c.d_model, c.n_heads, c.head_dim = shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim
@@ -122,6 +123,8 @@ def make_config(shape, max_ctx: Optional[int] = None, flags: int = 0, max_batch:
     for k in range(shape.K):
         c.topk[k] = shape.topk[k]
     c.flags = flags | (0 if getattr(shape, "use_sampled_token", True) else AMPH_FLAG_NO_SAMPLED_TOKEN)
+    c.temperature = float(temperature)
+    c.seed_lo, c.seed_hi = int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF
     return c
 
 
@@ -149,12 +152,12 @@ class Amphista:
 
     def __init__(self, shape, topo, weights: Dict[str, torch.Tensor], device="cuda:0",
                  max_ctx: Optional[int] = None, flags: int = 0, stream: Optional[torch.cuda.Stream] = None,
-                 max_batch: int = 1):
+                 max_batch: int = 1, temperature: float = 0.0, seed: int = 0):
         self.L = lib()
         self.shape, self.topo = shape, topo
         self.device = torch.device(device)
         self.B = int(max_batch)
-        self.cfg = make_config(shape, max_ctx, flags, max_batch)
+        self.cfg = make_config(shape, max_ctx, flags, max_batch, temperature, seed)
         self.tree = make_tree(topo)
         kvb, wsb = C.c_size_t(), C.c_size_t()
         self._check(self.L.amph_workspace_bytes(C.byref(self.cfg), C.byref(self.tree.c), C.byref(kvb), C.byref(wsb)), None)

@@ -53,7 +53,7 @@ struct Layout {
   size_t state_s, meta_s_, kv_tab_s, rope_s_, topk_ids_s, topk_vals_s, topk_cand_s, last_s, d_logits_s, att_o_s, att_ml_s;
   // shared
   size_t tree, inv_freq;
-  size_t tok, amax, override_tok, next_tok, amax_cand;                  // [Rcap] ints / candidates
+  size_t tok, amax, override_tok, next_tok, amax_cand, uniforms;        // [Rcap] ints / candidates / floats
   size_t x, hidden, h1, h2, pend_h, hp, attn_o;                           // fp32 rows
   size_t xn, q, att, act, cat, last_act, ao_act, aeb_act, lr_act;        // storage-type rows
   size_t partial, logits, ss_a, ss_b;
@@ -180,6 +180,7 @@ amph_status validate(const amph_config* c, const amph_tree* t, TreeDev* out) {
     if (c->topk[k] < 1 || c->topk[k] > kTopkStride || c->topk[k] > c->vocab)
       return fail(nullptr, AMPH_ERR_SHAPE, "topk[%d] = %d out of range 1..%d", k, c->topk[k], kTopkStride);
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 1.f)) return fail(nullptr, AMPH_ERR_SHAPE, "bad rms_eps / rope_theta");
+  if (!(c->temperature >= 0.f) || !(c->temperature < 1e6f)) return fail(nullptr, AMPH_ERR_SHAPE, "temperature must be 0 (greedy) or positive and finite");
   if (t->n_nodes < 1 || t->n_nodes > kMaxRows) return fail(nullptr, AMPH_ERR_SHAPE, "n_nodes must be in 1..%d", kMaxRows);
   if (!t->parent || !t->depth || !t->rank) return fail(nullptr, AMPH_ERR_INVALID_ARG, "tree arrays must not be NULL");
   if (c->max_batch * round_up(t->n_nodes < 16 ? 16 : t->n_nodes, 16) > kPrefillGroups * kMaxRows)
@@ -243,6 +244,7 @@ void make_layout(const amph_config& c, int n_nodes, Layout* L, int* Mcap_out, si
   l.override_tok = l.take(sizeof(int) * Rcap);
   l.next_tok = l.take(sizeof(int) * Rcap);
   l.amax_cand = l.take(2 * sizeof(float) * Rcap * 8);
+  l.uniforms = l.take(sizeof(float) * Rcap);
   l.x = l.take(4 * Rcap * d);
   l.hidden = l.take(4 * Rcap * d);
   l.h1 = l.take(4 * Rcap * d);
@@ -674,6 +676,19 @@ amph_status do_draft(amph_ctx* ctx, int32_t* out_ids, float* out_vals) {
   return rc;
 }
 
+// T > 0: replaces the greedy choices of every sequence's tree rows by draws from softmax(logits / T) (Section 2).
+void sample_tree_choices(amph_ctx* ctx) {
+  const Layout& l = ctx->lay;
+  const amph_config& c = ctx->cfg;
+  const unsigned long long seed = ((unsigned long long)c.seed_hi << 32) | c.seed_lo;
+  for (int b = 0; b < ctx->B; ++b) {
+    ProfScope p(ctx, AMPH_PROF_SELECT);
+    launch_sample_rows(ctx->at<float>(l.logits), c.vocab, b * ctx->Mver, ctx->tree_host.n_nodes, ctx->at<TreeDev>(l.tree),
+                       ctx->at<int>(l.tok) + b * ctx->Mver, ctx->state(b), b, 0, c.temperature, seed, ctx->at<int>(l.amax),
+                       ctx->at<float>(l.uniforms) + b * ctx->Mver, ctx->stream);
+  }
+}
+
 // tree_tokens / out_argmax: [B][n_nodes]
 amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_argmax) {
   const Layout& l = ctx->lay;
@@ -697,6 +712,7 @@ amph_status do_verify(amph_ctx* ctx, const int32_t* tree_tokens, int32_t* out_ar
   }
   target_forward(ctx, ps);
   target_head(ctx, ps.rows());
+  if (ctx->cfg.temperature > 0.f) sample_tree_choices(ctx);
   amph_status rc = AMPH_OK;
   for (int b = 0; b < B && rc == AMPH_OK && out_argmax; ++b)
     rc = copy_out(ctx, out_argmax + (size_t)b * N, ctx->at<int>(l.amax) + b * ctx->Mver, sizeof(int) * N);
@@ -938,6 +954,9 @@ amph_status amph_prefill_seq(amph_ctx* ctx, int32_t seq, const int32_t* prompt_i
       }
       run_sals(ctx, ctx->at<float>(l.hidden), next_tok, pss);
     }
+    if (last && c.temperature > 0.f)        // the token after the prompt is drawn, not the arg-max (stream 1 of the generator, step 0)
+      launch_sample_rows(ctx->at<float>(l.logits), c.vocab, cnt - 1, 1, nullptr, nullptr, ctx->state(seq), seq, 1, c.temperature,
+                         ((unsigned long long)c.seed_hi << 32) | c.seed_lo, ctx->at<int>(l.amax), nullptr, st);
     if (last)
       launch_prefill_tail(ctx->state(seq), ctx->at<int>(l.amax), cnt - 1, ctx->at<float>(l.hidden),
                           ctx->at<float>(l.pend_h) + (size_t)seq * kSmallRows * c.d_model, c.d_model, n, st);
@@ -1069,6 +1088,7 @@ amph_status amph_get_tensor(amph_ctx* ctx, const char* name, void* dst, size_t b
       {"sal_h", l.last + l.last_s * seq, 4 * 2 * d},
       {"tree_tokens", l.tok + 4 * seq * Mv, 4 * N},
       {"argmax", l.amax + 4 * seq * Mv, 4 * N},
+      {"uniforms", l.uniforms + 4 * seq * Mv, 4 * N},
   };
   for (auto& p : plain) {
     if (nm == p.n) {
@@ -1112,6 +1132,17 @@ amph_status amph_set_tensor(amph_ctx* ctx, const char* name, const void* src, si
     return rc;
   }
   if (ctx->phase != PH_VERIFIED) return fail(ctx, AMPH_ERR_STATE, "amph_set_tensor must follow amph_verify_tree");
+  if (nm == "logits") {                          // T > 0: replace the verified rows' logits and draw the choices again
+    const amph_config& c = ctx->cfg;
+    const size_t N = ctx->tree_host.n_nodes;
+    if (!(c.temperature > 0.f)) return fail(ctx, AMPH_ERR_STATE, "'logits' can be set with temperature > 0 only");
+    if (bytes != sizeof(float) * N * c.vocab) return fail(ctx, AMPH_ERR_INVALID_ARG, "'logits' takes exactly n_nodes * vocab floats");
+    amph_status rc = cuda_check(ctx, cudaMemcpyAsync(ctx->at<float>(ctx->lay.logits) + (size_t)seq * ctx->Mver * c.vocab, src, bytes,
+                                                     cudaMemcpyDefault, ctx->stream), "set_tensor");
+    if (rc != AMPH_OK) return rc;
+    sample_tree_choices(ctx);
+    return finish(ctx, "sampling");
+  }
   size_t off;
   if (nm == "tree_tokens") off = ctx->lay.tok;
   else if (nm == "argmax") off = ctx->lay.amax;

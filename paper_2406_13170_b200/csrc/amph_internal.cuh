@@ -51,6 +51,7 @@ struct DevState {
   int next_root;
   int path[16];
   int out_tok[16];
+  int step;                 // acceptances this sequence has seen (counter of the sampling generator)
 };
 
 // Programmatic dependent launch.  Every kernel of the step is launched with the attribute below, so it
@@ -211,6 +212,14 @@ void launch_meta_pending(RowMeta* meta, const DevState* s, cudaStream_t st);    
 void launch_tree_build(const TreeDev* tree, DevState* s, const int* topk_ids, const int* override_tok,
                        int* tok, RowMeta* meta, cudaStream_t st);
 void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st);
+// Sampling at temperature T > 0 (Table 2): choice[r] for rows row0 .. row0 + n_rows - 1 = the token the target draws after
+// that row from softmax(logits / T) with the row's own uniform (Philox4x32-10 keyed by seed; counter = row - row0, the
+// sequence's step count, seq, stream).  With a tree (tok != NULL) the vocabulary is walked in the order (tokens of the
+// row's children in node order, then every other id ascending), so that a child is accepted iff its token is the choice:
+// the rejection-sampling test of Section 2 for point-mass proposals.  uniforms_out (may be NULL) receives the uniforms.
+void launch_sample_rows(const float* logits, int vocab, int row0, int n_rows, const TreeDev* tree, const int* tok,
+                        const DevState* s, int seq, int stream_id, float temperature, unsigned long long seed, int* choice,
+                        float* uniforms_out, cudaStream_t st);
 void launch_compact(const DevState* s, const KvView* kv_layers, int n_layers, int dtype, int n_heads,
                     int head_dim, int max_ctx, const float* hidden, float* pend_h, int d, cudaStream_t st);
 void launch_reduce_partials(PartialView P, float* y, int rows, int cols, cudaStream_t st);

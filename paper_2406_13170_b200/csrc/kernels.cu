@@ -1027,11 +1027,149 @@ __global__ void accept_kernel(const TreeDev* __restrict__ tree, DevState* s, con
     s->C = C + L;
     s->root = nr;
     s->n_pending = L;
+    s->step += 1;
   }
 }
 
 void launch_accept(const TreeDev* tree, DevState* s, const int* tok, const int* amax, cudaStream_t st) {
   launch_pdl(accept_kernel, dim3(1), dim3(kMaxRows), 0, st, tree, s, tok, amax);
+}
+
+// --------------------------------------------------------------------------------------------
+// Sampling at a temperature (Table 2; Section 2, rejection sampling with point-mass proposals)
+// --------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds; each multiplies counter words 0 and 2 by fixed odd constants,
+// crosses the halves of the 64-bit products and mixes in the key, which is bumped by Weyl constants between rounds.
+__device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = h1 ^ c1 ^ k0, n2 = h0 ^ c3 ^ k1;
+    c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+  }
+  return c0;
+}
+
+constexpr int kSampleThreads = 1024;
+constexpr int kSampleMaxChildren = 16;       // candidates a head keeps at most = children a node has at most
+
+// One block per row.  w(v) = exp((l_v - max) / T); the row's uniform scaled by the sum of all weights is compared with
+// running sums of w, so nothing is divided.  Sums are taken in a fixed order (deterministic).
+__global__ void __launch_bounds__(kSampleThreads)
+sample_rows_kernel(const float* __restrict__ logits, int vocab, int row0, const TreeDev* __restrict__ tree,
+                   const int* __restrict__ tok, const DevState* __restrict__ s, int seq, int stream_id, float inv_t,
+                   uint32_t k0, uint32_t k1, int* __restrict__ choice, float* __restrict__ uniforms_out) {
+  pdl_wait();
+  pdl_launch_dependents();
+  __shared__ float red[kSampleThreads / 32];
+  __shared__ float part[kSampleThreads];
+  __shared__ int kid_tok[kSampleMaxChildren];
+  __shared__ int n_kids_s, result_s;
+  __shared__ float target_s, base_s;
+  const int r = blockIdx.x, row = row0 + r, tid = threadIdx.x;
+  const float* l = logits + (size_t)row * vocab;
+  // row maximum
+  float m = -INFINITY;
+  for (int v = tid; v < vocab; v += kSampleThreads) m = fmaxf(m, l[v]);
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  m = red[0];
+  for (int i = 1; i < kSampleThreads / 32; ++i) m = fmaxf(m, red[i]);
+  __syncthreads();
+  // the distinct tokens of the row's children, in node order
+  if (tid == 0) {
+    int nk = 0;
+    if (tree != nullptr && tok != nullptr) {
+      const int N = tree->n_nodes;
+      for (int c = r + 1; c < N && nk < kSampleMaxChildren; ++c) {
+        if (tree->parent[c] != r) continue;
+        const int x = tok[c];
+        bool seen = x < 0 || x >= vocab;
+        for (int j = 0; j < nk; ++j) seen = seen || kid_tok[j] == x;
+        if (!seen) kid_tok[nk++] = x;
+      }
+    }
+    n_kids_s = nk;
+    result_s = -1;
+  }
+  __syncthreads();
+  const int nk = n_kids_s;
+  // every thread owns a contiguous range of ids; its weight sum leaves the children's tokens out
+  const int chunk = (vocab + kSampleThreads - 1) / kSampleThreads;
+  const int lo = tid * chunk, hi = lo + chunk < vocab ? lo + chunk : vocab;
+  float mine = 0.f;
+  for (int v = lo; v < hi; ++v) {
+    bool kid = false;
+    for (int j = 0; j < nk; ++j) kid = kid || kid_tok[j] == v;
+    if (!kid) mine += __expf((l[v] - m) * inv_t);
+  }
+  part[tid] = mine;
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t w = philox_first_word((uint32_t)r, (uint32_t)s->step, (uint32_t)seq, (uint32_t)stream_id, k0, k1);
+    const float u = (float)(w >> 8) * (1.0f / 16777216.0f);
+    if (uniforms_out) uniforms_out[r] = u;
+    float kids = 0.f, rest = 0.f;
+    float wk[kSampleMaxChildren];
+    for (int j = 0; j < nk; ++j) { wk[j] = __expf((l[kid_tok[j]] - m) * inv_t); kids += wk[j]; }
+    for (int i = 0; i < kSampleThreads; ++i) rest += part[i];
+    const float target = u * (kids + rest);
+    float acc = 0.f;
+    int res = -1;
+    for (int j = 0; j < nk && res < 0; ++j) {            // children first: accepted iff the running sum passes the target
+      acc += wk[j];
+      if (target < acc) res = kid_tok[j];
+    }
+    result_s = res;
+    target_s = target;
+    base_s = kids;
+  }
+  __syncthreads();
+  if (result_s >= 0) {
+    if (tid == 0) choice[row] = result_s;
+    return;
+  }
+  // residual distribution: the first id, ascending, children's tokens left out, whose running sum exceeds the target
+  if (tid == 0) {
+    float acc = base_s;
+    int owner = -1;
+    for (int i = 0; i < kSampleThreads; ++i) {
+      if (acc + part[i] > target_s && part[i] > 0.f) { owner = i; break; }
+      acc += part[i];
+    }
+    if (owner < 0) {                                       // rounding left the target above the total: the last admissible id
+      for (int i = kSampleThreads - 1; i >= 0 && owner < 0; --i)
+        if (part[i] > 0.f) { owner = i; acc = -INFINITY; }   // its walk then ends on its last admissible id
+    }
+    n_kids_s = nk;
+    result_s = -2 - owner;                                 // owner thread, encoded
+    base_s = acc;
+  }
+  __syncthreads();
+  const int owner = -2 - result_s;
+  if (tid == owner) {
+    float acc = base_s;
+    int res = -1, last = -1;
+    for (int v = lo; v < hi; ++v) {
+      bool kid = false;
+      for (int j = 0; j < nk; ++j) kid = kid || kid_tok[j] == v;
+      if (kid) continue;
+      last = v;
+      acc += __expf((l[v] - m) * inv_t);
+      if (acc > target_s) { res = v; break; }
+    }
+    choice[row] = res >= 0 ? res : last;
+  }
+}
+
+void launch_sample_rows(const float* logits, int vocab, int row0, int n_rows, const TreeDev* tree, const int* tok,
+                        const DevState* s, int seq, int stream_id, float temperature, unsigned long long seed, int* choice,
+                        float* uniforms_out, cudaStream_t st) {
+  launch_pdl(sample_rows_kernel, dim3(n_rows), dim3(kSampleThreads), 0, st, logits, vocab, row0, tree, tok, s, seq, stream_id,
+             1.0f / temperature, (uint32_t)(seed & 0xffffffffull), (uint32_t)(seed >> 32), choice, uniforms_out);
 }
 
 // Block l < n_layers moves layer l's accepted key / value rows: slot C_old + j <- C_old + path[j].
@@ -1122,6 +1260,7 @@ __global__ void prefill_tail_kernel(DevState* s, const int* __restrict__ amax, i
     s->C_old = C;
     s->best = 0;
     s->next_root = root;
+    s->step = 0;
   }
 }
 
