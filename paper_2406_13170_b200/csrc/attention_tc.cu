@@ -153,6 +153,12 @@ __device__ __forceinline__ void tmem_ld_frag64(uint32_t taddr, uint32_t* v) {
                : "r"(taddr)
                : "memory");
 }
+// 2^x on the special-function unit: ex2(-inf) = +0, so masked scores need no test of their own
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -432,18 +438,21 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
       tmax_b = fmaxf(tmax_b, __shfl_xor_sync(0xffffffffu, tmax_b, 1));
       tmax_b = fmaxf(tmax_b, __shfl_xor_sync(0xffffffffu, tmax_b, 2));
       const float mn_a = fmaxf(m_a, tmax_a), mn_b = fmaxf(m_b, tmax_b);
-      const float ca = mn_a == -INFINITY ? 1.f : exp2f(m_a - mn_a);
-      const float cb = mn_b == -INFINITY ? 1.f : exp2f(m_b - mn_b);
+      // a row that has seen no visible key yet (m = -inf) holds zeros: any finite factor will do
+      const float ca = m_a == -INFINITY ? 1.f : ex2_approx(m_a - mn_a);
+      const float cb = m_b == -INFINITY ? 1.f : ex2_approx(m_b - mn_b);
+      if (ca != 1.f || cb != 1.f) {                    // the running maximum moved: bring the running output to the new scale
 #pragma unroll
-      for (int i = 0; i < DH / 2; ++i) acc[i] *= ((i >> 1) & 1) ? cb : ca;
+        for (int i = 0; i < DH / 2; ++i) acc[i] *= ((i >> 1) & 1) ? cb : ca;
+      }
+      const float sub_a = mn_a == -INFINITY ? 0.f : mn_a, sub_b = mn_b == -INFINITY ? 0.f : mn_b;
       float ps_a = 0.f, ps_b = 0.f;
 #pragma unroll
       for (int rep = 0; rep < kChunk / 8; ++rep) {
         float p[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float v = s[rep * 4 + e];
-          p[e] = v == -INFINITY ? 0.f : exp2f(v - (e < 2 ? mn_a : mn_b));
+          p[e] = ex2_approx(s[rep * 4 + e] - (e < 2 ? sub_a : sub_b));
         }
         ps_a += p[0] + p[1];
         ps_b += p[2] + p[3];
