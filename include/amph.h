@@ -298,7 +298,11 @@ amph_status amph_selftest_wait_timeout(const void* x_dev, int32_t x_rows_cap, co
  * Limit: 256 + (rows rounded up to 16) * n_seg * out * 4 bytes must not exceed
  * AMPH_NOALLOC_SCRATCH_BYTES, otherwise AMPH_ERR_WORKSPACE (nothing is launched).
  * The first call on each device looks up the array's device address (with that device current);
- * make that first call before starting any stream capture.  All calls on a device share the one
+ * make that first call before starting any stream capture.  With CUDA's default lazy module loading the
+ * library's device image, and with it the array's 16 MiB, is placed on a device the first time the
+ * library is used there, which may be this first call: make it while the device still has that much
+ * memory free (before another component takes all of it), or run the process with CUDA_MODULE_LOADING=EAGER;
+ * otherwise the first call can fail with AMPH_ERR_CUDA.  All calls on a device share the one
  * array, which keeps the previous call's contents (the call clears what must start at zero): calls
  * whose kernels may overlap on the GPU (different streams, or several threads) race on it, so
  * serialise them.  Stream-ordered; y_dev is valid once the stream has been synchronised. */

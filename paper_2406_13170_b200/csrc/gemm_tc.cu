@@ -796,6 +796,15 @@ bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, 
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }
 
+void tc_gemm_rebind(TcGemm* g, int xb, void* ptr, int rows, int cols, int* err_flag) {
+  if (!g || xb < 0 || xb >= g->n_x) return;
+  g->xptr[xb] = ptr;
+  g->xrows[xb] = rows;
+  g->xcols[xb] = cols;
+  g->err_flag = err_flag;
+  if (g->cache.size() > 512) g->cache.clear();          // a long-lived plan set must not grow without bound
+}
+
 void tc_gemm_set_selftest(TcGemm* g, unsigned long long wait_limit_ns, unsigned extra_tx) {
   g->wait_limit_ns = wait_limit_ns;
   g->extra_tx = extra_tx;

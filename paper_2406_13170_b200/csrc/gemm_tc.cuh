@@ -38,6 +38,10 @@ bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, 
 
 void tc_gemm_destroy(TcGemm* g);
 
+// Points activation buffer `xb` of an existing plan set at another bf16 [rows][cols] buffer and the error flag at
+// another device int (host-side bookkeeping only; tensor maps of buffers seen before stay cached, up to a bound).
+void tc_gemm_rebind(TcGemm* g, int xb, void* ptr, int rows, int cols, int* err_flag);
+
 // Failure-path self-test: every barrier wait of later launches gives up after wait_limit_ns, and the first stage's
 // barrier of each CTA expects extra_tx bytes more than its copies deliver (so that wait can never complete).
 void tc_gemm_set_selftest(TcGemm* g, unsigned long long wait_limit_ns, unsigned extra_tx);

@@ -25,6 +25,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 std::mutex g_setup_mutex;
 void* g_scratch_addr[kMaxDevices];     // device address of g_static_scratch, per device ordinal
+TcGemm* g_plans[kMaxDevices];          // tensor-core plan set per device, created by the first tensor-core call and kept
 
 // In host code `g_static_scratch` is only a handle of the symbol, not an address a kernel may
 // dereference: the device address has to be looked up, once per device, with that device current.
@@ -104,12 +105,18 @@ amph_status amph_project_noalloc(const void* x_dev, int32_t x_rows_cap, const vo
     if (dtype != AMPH_DTYPE_BF16) { say(err_msg, err_len, "the tensor-core kernel takes bf16 only"); return AMPH_ERR_SHAPE; }
     void* xb[1] = {const_cast<void*>(x_dev)};
     const int xr[1] = {x_rows_cap}, xc[1] = {in};
-    TcGemm* g = tc_gemm_create(xb, xr, xc, 1, err);        // host-side bookkeeping only
+    // The plan set (driver entry point, kernel attributes, cached tensor maps: host-side bookkeeping only) is made
+    // once per device and re-pointed at this call's activations, so a steady-state call encodes at most one new map.
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    TcGemm*& g = g_plans[dev];
+    if (!g) g = tc_gemm_create(xb, xr, xc, 1, err);
     if (!g) { say(err_msg, err_len, "tensor-map encoder unavailable or not an sm_100 device"); return AMPH_ERR_CUDA; }
+    tc_gemm_rebind(g, 0, xb[0], xr[0], xc[0], err);
     int splits = 0;
     size_t stride = 0;
     const bool ok = tc_gemm_launch(g, 0, w, n_seg, out, in, rows, P, p_floats, &splits, &stride, st);
-    tc_gemm_destroy(g);
     if (!ok) { say(err_msg, err_len, "shape not covered by the tensor-core kernel"); return AMPH_ERR_SHAPE; }
     pv.splits = splits;
     pv.split_stride = stride;

@@ -50,3 +50,23 @@ def test_noalloc_rejects_oversized_projection():
     with pytest.raises(AmphError) as e:
         project_noalloc(x, [w, w, w, w], 128, False, y)          # 128 x 128000 fp32 = 65 MB > 16 MiB
     assert e.value.status == 5 and "limit" in str(e.value)
+
+
+def test_noalloc_at_the_exact_size_limit():
+    """16 padded rows x 262140 features x 4 bytes + the 256-byte header is exactly the built-in 16 MiB: accepted and
+    correct; one more row (padded to 32) no longer fits and is refused before anything is launched."""
+    from paper_2406_13170_b200 import project, project_noalloc, AmphError
+    dev = "cuda:0"
+    out, in_ = 262140, 64
+    assert 256 + 16 * out * 4 == 16 << 20
+    w = inputs.normal_tensor((out, in_), 0.02, 21, "w", dtype=torch.bfloat16, device=dev)
+    x = inputs.normal_tensor((32, in_), 1.0, 21, "x", dtype=torch.bfloat16, device=dev)
+    y = torch.full((16, out), float("nan"), dtype=torch.float32, device=dev)
+    project_noalloc(x, [w], 16, False, y)
+    torch.cuda.synchronize()
+    ref = project(x, [w], 16, False)
+    assert float((y - ref).abs().max()) <= TOL * max(1.0, float(ref.abs().max()))
+    y17 = torch.zeros(17, out, dtype=torch.float32, device=dev)
+    with pytest.raises(AmphError) as e:
+        project_noalloc(x, [w], 17, False, y17)
+    assert e.value.status == 5
