@@ -419,13 +419,13 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
       chunk_visibility(mb0, mb1, live_b, base - key0, 2 * qd, vb0, vb1);
       if (base - key0 >= kChunk && live_a && live_b) {                       // committed context: nothing is masked
 #pragma unroll
-        for (int i = 0; i < kChunk / 2; ++i) s[i] = __uint_as_float(sr[i]) * scale_log2;
+        for (int i = 0; i < kChunk / 2; ++i) s[i] = __uint_as_float(sr[i]);
       } else {
 #pragma unroll
         for (int i = 0; i < kChunk / 2; ++i) {
           const int bit = 8 * (i >> 2) + (i & 1);                            // column of this register minus 2 qd
           const u64 w = ((i >> 1) & 1) ? (bit < 64 ? vb0 : vb1) : (bit < 64 ? va0 : va1);
-          s[i] = ((w >> (bit & 63)) & 1ull) ? __uint_as_float(sr[i]) * scale_log2 : -INFINITY;       // base-2 logits
+          s[i] = ((w >> (bit & 63)) & 1ull) ? __uint_as_float(sr[i]) : -INFINITY;       // raw scores; the scale joins the exponent below
         }
       }
 #pragma unroll
@@ -437,7 +437,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
       tmax_a = fmaxf(tmax_a, __shfl_xor_sync(0xffffffffu, tmax_a, 2));
       tmax_b = fmaxf(tmax_b, __shfl_xor_sync(0xffffffffu, tmax_b, 1));
       tmax_b = fmaxf(tmax_b, __shfl_xor_sync(0xffffffffu, tmax_b, 2));
-      const float mn_a = fmaxf(m_a, tmax_a), mn_b = fmaxf(m_b, tmax_b);
+      const float mn_a = fmaxf(m_a, tmax_a * scale_log2), mn_b = fmaxf(m_b, tmax_b * scale_log2);     // base-2 logits
       // a row that has seen no visible key yet (m = -inf) holds zeros: any finite factor will do
       const float ca = m_a == -INFINITY ? 1.f : ex2_approx(m_a - mn_a);
       const float cb = m_b == -INFINITY ? 1.f : ex2_approx(m_b - mn_b);
@@ -452,7 +452,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
         float p[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          p[e] = ex2_approx(s[rep * 4 + e] - (e < 2 ? sub_a : sub_b));
+          p[e] = ex2_approx(fmaf(s[rep * 4 + e], scale_log2, -(e < 2 ? sub_a : sub_b)));
         }
         ps_a += p[0] + p[1];
         ps_b += p[2] + p[3];

@@ -197,3 +197,37 @@ def test_low_temperature_is_greedy_on_the_gpu():
         outs.append(out)
         model.close()
     assert outs[0] == outs[1]
+
+
+def test_sampling_in_a_batch_uses_one_generator_stream_per_sequence():
+    """Two sequences with the SAME prompt at T = 0.7: sequence 0 draws what a single-sequence context with that seed
+    draws (its uniforms are keyed by sequence index 0), sequence 1 has uniforms of its own and soon emits other tokens;
+    the uniforms tap of each sequence equals the oracle's generator for that sequence index."""
+    from paper_2406_13170_b200 import Amphista
+    shape = inputs.get_shape("tiny")
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    w = inputs.make_weights(shape, seed=0, init="fan_in")
+    w_gpu = {k: v.to("cuda:0") for k, v in w.items()}
+    prompt = inputs.make_prompt(shape).tolist()
+    K, N = shape.K, topo.n_nodes
+
+    def run(batch):
+        model = Amphista(shape, topo, w_gpu, temperature=0.7, seed=SEED, max_batch=batch)
+        out = [[model.prefill(prompt, seq=b)] for b in range(batch)]
+        tok = torch.zeros(batch, K + 1, dtype=torch.int32, device="cuda:0")
+        n = torch.zeros(batch, dtype=torch.int32, device="cuda:0")
+        for step in range(5):
+            model.draft(); model.verify_tree()
+            for b in range(batch):
+                assert model.get_tensor(f"uniforms#{b}", (N,)).cpu().tolist() == sm.node_uniforms(SEED, step, b, N)
+            model.accept(tok, n)
+            torch.cuda.synchronize()
+            for b in range(batch):
+                out[b] += tok[b, :int(n[b])].tolist()
+        model.close()
+        return out
+
+    single = run(1)[0]
+    both = run(2)
+    assert both[0] == single
+    assert both[1] != both[0]
