@@ -454,12 +454,36 @@ bool layer_forward(amph_ctx* ctx, const LayerW& w, CacheOf cache_of, float* x, c
     if (!fused_rope) cudaGetLastError();
   }
   if (!fused_rope) P = project(ctx, XB_XN, qkv, 3, c.d_model, c.d_model, rows);
-  for (int g = 0; g < ps.G && !fused_rope; ++g) {     // rotary embedding + cache write, per group (its own cache and slots)
+  bool grouped_rope = false;
+  if (!fused_rope && ps.G > 1) {                      // every group's rotary embedding + cache write in one launch
+    ProfScope p(ctx, AMPH_PROF_ROPE_KV);
+    RopeGroups gr;
+    gr.G = ps.G;
+    gr.rpg = ps.rpg;
+    for (int g = 0; g < ps.G; ++g) {
+      const KvView kv = cache_of(ps.seq[g]);
+      gr.meta[g] = ps.meta[g]; gr.rope[g] = ps.rope[g]; gr.kc[g] = kv.k; gr.vc[g] = kv.v;
+    }
+    launch_qkv_rope_groups(P, gr, ctx->ws + l.q, ctx->dtype, c.n_heads, c.head_dim, c.max_ctx, st, rs);
+    grouped_rope = true;
+  }
+  for (int g = 0; g < ps.G && !fused_rope && !grouped_rope; ++g) {     // rotary embedding + cache write, per group (its own cache and slots)
     ProfScope p(ctx, AMPH_PROF_ROPE_KV);
     launch_qkv_rope(rows_from(P, g * ps.rpg), ps.meta[g], ps.rope[g], ctx->ws + l.q + ctx->esz * g * ps.rpg * d, cache_of(ps.seq[g]),
                     ctx->dtype, ps.rpg, c.n_heads, c.head_dim, c.max_ctx, st, rows_from(rs, g * ps.rpg));
   }
-  for (int g = 0; g < ps.G; ++g) {                    // tree attention, per group
+  bool grouped_attn = false;
+  if (ctx->attn_tc && ps.G > 1 && !(c.flags & AMPH_FLAG_SEPARATE_MERGE)) {   // every group's tree attention in one launch
+    ProfScope p(ctx, AMPH_PROF_ATTENTION);
+    KvView kvs[kMaxSeq];
+    int keys = 0;
+    for (int g = 0; g < ps.G; ++g) { kvs[g] = cache_of(ps.seq[g]); keys = ps.keys[g] > keys ? ps.keys[g] : keys; }
+    const int splits = attn_tc_splits(ctx->attn_tc, keys, c.n_heads, ps.rpg, l.attn_splits);
+    grouped_attn = launch_tree_attention_tc_groups(ctx->attn_tc, ctx->ws + l.q, ctx->Rcap, ps.G, kvs, ps.meta, ps.rpg, c.n_heads,
+                                                   c.head_dim, c.max_ctx, splits, keys, st, ctx->ws + l.att, &ctx->state(0)->err);
+    if (!grouped_attn) cudaGetLastError();
+  }
+  for (int g = 0; g < ps.G && !grouped_attn; ++g) {   // tree attention, per group
     ProfScope p(ctx, AMPH_PROF_ATTENTION);
     const KvView kv = cache_of(ps.seq[g]);
     AttnScratch sc = {ctx->grp<float>(l.att_o, l.att_o_s, g), ctx->grp<float>(l.att_ml, l.att_ml_s, g)};

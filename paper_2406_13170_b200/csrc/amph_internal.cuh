@@ -149,6 +149,16 @@ void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, voi
                      int dtype, int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st,
                      RowScale rs = RowScale());
 
+struct RopeGroups {         // per row group: row table, rotary table, cache
+  const RowMeta* meta[AMPH_MAX_BATCH];
+  const float2* rope[AMPH_MAX_BATCH];
+  void* kc[AMPH_MAX_BATCH];
+  void* vc[AMPH_MAX_BATCH];
+  int G, rpg;
+};
+void launch_qkv_rope_groups(PartialView P, const RopeGroups& gr, void* q, int dtype, int n_heads, int head_dim, int max_ctx,
+                            cudaStream_t st, RowScale rs = RowScale());
+
 struct AttnScratch {
   float* o;                 // [splits][heads][rows][head_dim]
   float* ml;                // [splits][heads][rows][2]  (running max, running sum)
@@ -174,6 +184,10 @@ int attn_tc_stages(int keys_bound, int splits, int head_dim);
 bool launch_tree_attention_tc(AttnTc* a, const void* q, int q_rows_cap, KvView kv, const RowMeta* meta, AttnScratch sc, int rows,
                               int n_heads, int head_dim, int max_ctx, int splits, int keys_bound, cudaStream_t st,
                               void* merged_out, int* err_flag);
+
+bool launch_tree_attention_tc_groups(AttnTc* a, const void* q, int q_rows_cap, int G, const KvView* kv, const RowMeta* const* meta,
+                                     int rows, int n_heads, int head_dim, int max_ctx, int splits, int keys_bound, cudaStream_t st,
+                                     void* merged_out, int* err_flag);
 
 void launch_swiglu(PartialView P, void* act, int dtype, int rows, int f, cudaStream_t st, RowScale rs = RowScale(),
                    int early = 0);

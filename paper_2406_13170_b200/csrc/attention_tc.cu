@@ -39,13 +39,21 @@ constexpr int kTmemCols = 256;       // S in columns [0, 128), O in [128, 128 + 
                                      // become resident beside this kernel and allocate their accumulators
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
+constexpr int kMaxGroups = AMPH_MAX_BATCH;   // row groups (sequences, or chunks of one prompt) one launch may carry
+
+// NG = 1 for the usual launch (kernel parameters stay small: they are copied with every launch), kMaxGroups for the grouped one
+template <int NG>
 struct AttnMaps {
-  CUtensorMap q, k, v;
+  CUtensorMap q;                      // all groups' query rows: group g starts at row g * rows_per_group
+  CUtensorMap k[NG], v[NG];           // the cache each group reads
 };
 
+template <int NG>
 struct AttnParams {
-  const RowMeta* meta;
-  float* po;                 // partial outputs / (max, sum) for the separate merge
+  const RowMeta* meta[NG];
+  int nrb, rpg;              // 64-row blocks per group (grid.z = groups * nrb), rows per group
+  int same_cache;            // the groups are consecutive chunks of one sequence: slots from meta[0]->base on are written by this pass
+  float* po;                 // partial outputs / (max, sum) for the separate merge (one group only)
   float* pml;
   bf16* out;                 // merged output rows (cluster merge), or NULL
   int rows_cap, n_heads, max_ctx, stages;
@@ -198,9 +206,9 @@ __device__ __forceinline__ void chunk_visibility(u64 m0, u64 m1, bool live, int 
   v1 = a1 >> sh;
 }
 
-template <int DH, bool MERGE>
+template <int DH, bool MERGE, int NG>
 __global__ void __launch_bounds__(kThreads, 2)
-tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm) {
+tree_attn_tc_kernel(const __grid_constant__ AttnMaps<NG> maps, const AttnParams<NG> prm) {
   constexpr int NB = DH / 64;                        // 64-wide blocks of the head dimension (one 128-byte swizzle row each)
   constexpr uint32_t kQBlock = kRows * 128;          // bytes of one Q / P block: 64 rows x 128 bytes
   constexpr uint32_t kKvBlock = kChunk * 128;        // bytes of one K / V block: 128 keys x 128 bytes
@@ -212,7 +220,10 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.x, split = blockIdx.y, rb = blockIdx.z;
+  const int h = blockIdx.x, split = blockIdx.y;
+  const int grp = NG == 1 ? 0 : (int)blockIdx.z / prm.nrb, rb = NG == 1 ? (int)blockIdx.z : (int)blockIdx.z - grp * prm.nrb;
+  const RowMeta* const meta = prm.meta[grp];
+  const int row_base = grp * prm.rpg;                // first row of this group in the query / output buffers
   const int stages = prm.stages;
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* Qs = smem;
@@ -239,7 +250,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
 
   // The row table was written several kernels ago (every kernel between it and this one waits for its own
   // predecessor before it lets its successor start), so it may be read before the dependency wait.
-  const int base = prm.meta->base, n_rows = prm.meta->n_rows;
+  const int base = meta->base, n_rows = meta->n_rows;
   const int total = base + n_rows;
   int len = (total + (int)gridDim.y - 1) / (int)gridDim.y;
   len = (len + kChunk - 1) / kChunk * kChunk;          // whole chunks: a chunk never straddles two splits
@@ -263,19 +274,22 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
     const bool leader = elect_one();
     if (leader) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.q) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.k) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.v) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.k[grp]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.v[grp]) : "memory");
     }
     int issued = 0;
     bool k_only = false;                               // gave up between the key and the value copies of chunk `issued`
     // committed context: nothing the previous kernel writes
     if (leader) {
-      while (issued < n_chunks && issued < stages && s_lo + (issued + 1) * kChunk <= base) {
+      // slots the kernel before this one may still be writing must wait: everything from this group's base on, and, when
+      // the groups are chunks of one prompt, everything from the first group's base on (earlier chunks of the same pass)
+      const int settled = (NG > 1 && prm.same_cache) ? prm.meta[0]->base : base;
+      while (issued < n_chunks && issued < stages && s_lo + (issued + 1) * kChunk <= settled) {
         uint8_t* kdst = St + (size_t)issued * kStage;
         mbar_expect_tx(&k_full[issued], NB * kKvBlock);
         mbar_expect_tx(&v_full[issued], NB * kKvBlock);
-        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + j * kKvBlock, &maps.k, 64 * j, s_lo + issued * kChunk, h, &k_full[issued]);
-        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + (NB + j) * kKvBlock, &maps.v, 64 * j, s_lo + issued * kChunk, h, &v_full[issued]);
+        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + j * kKvBlock, &maps.k[grp], 64 * j, s_lo + issued * kChunk, h, &k_full[issued]);
+        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + (NB + j) * kKvBlock, &maps.v[grp], 64 * j, s_lo + issued * kChunk, h, &v_full[issued]);
         ++issued;
       }
     }
@@ -284,7 +298,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
     pdl_launch_dependents();
     if (leader && n_chunks > 0) {
       mbar_expect_tx(&q_full, NB * kQBlock);
-      for (int j = 0; j < NB; ++j) tma_load_2d(Qs + j * kQBlock, &maps.q, h * DH + 64 * j, rb * kRows, &q_full);
+      for (int j = 0; j < NB; ++j) tma_load_2d(Qs + j * kQBlock, &maps.q, h * DH + 64 * j, row_base + rb * kRows, &q_full);
     }
     for (int c = issued; c < n_chunks; ++c) {
       const int st = c % stages, round = c / stages;
@@ -294,13 +308,13 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
       if (round > 0 && !__all_sync(0xffffffffu, mbar_wait(&k_empty[st], (round & 1) ^ 1, &abort_flag))) break;
       if (leader) {
         mbar_expect_tx(&k_full[st], NB * kKvBlock);
-        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + j * kKvBlock, &maps.k, 64 * j, s_lo + c * kChunk, h, &k_full[st]);
+        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + j * kKvBlock, &maps.k[grp], 64 * j, s_lo + c * kChunk, h, &k_full[st]);
       }
       __syncwarp();
       if (round > 0 && !__all_sync(0xffffffffu, mbar_wait(&v_empty[st], (round & 1) ^ 1, &abort_flag))) { k_only = true; break; }
       if (leader) {
         mbar_expect_tx(&v_full[st], NB * kKvBlock);
-        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + (NB + j) * kKvBlock, &maps.v, 64 * j, s_lo + c * kChunk, h, &v_full[st]);
+        for (int j = 0; j < NB; ++j) tma_load_3d(kdst + (NB + j) * kKvBlock, &maps.v[grp], 64 * j, s_lo + c * kChunk, h, &v_full[st]);
       }
       __syncwarp();
       issued = c + 1;
@@ -380,8 +394,8 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
     const int ga = rb * kRows + row_a, gb = ga + 8;
     const bool live_a = ga < n_rows, live_b = gb < n_rows;
     u64 ma0 = 0, ma1 = 0, mb0 = 0, mb1 = 0;
-    if (live_a) { ma0 = prm.meta->mask[ga][0]; ma1 = prm.meta->mask[ga][1]; }
-    if (live_b) { mb0 = prm.meta->mask[gb][0]; mb1 = prm.meta->mask[gb][1]; }
+    if (live_a) { ma0 = meta->mask[ga][0]; ma1 = meta->mask[ga][1]; }
+    if (live_b) { mb0 = meta->mask[gb][0]; mb1 = meta->mask[gb][1]; }
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     auto add_output = [&]() {                          // acc += O of the chunk whose P V has completed
@@ -543,7 +557,7 @@ tree_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnParams prm)
         uint2 u;
         u.x = pack_bf16(a.x * inv, a.y * inv);
         u.y = pack_bf16(a.z * inv, a.w * inv);
-        *reinterpret_cast<uint2*>(prm.out + (size_t)gr * prm.n_heads * DH + h * DH + lane * 4) = u;
+        *reinterpret_cast<uint2*>(prm.out + (size_t)(row_base + gr) * prm.n_heads * DH + h * DH + lane * 4) = u;
       }
     }
     cluster_sync_all();                                // nobody leaves while a peer may still read its shared memory
@@ -647,22 +661,31 @@ int attn_tc_stages(int keys_bound, int splits, int head_dim) {
 
 namespace {
 
-template <int DH>
-bool launch_t(AttnTc* a, const void* q, int q_rows_cap, KvView kv, const RowMeta* meta, AttnScratch sc, int rows, int n_heads,
-              int max_ctx, int splits, int keys_bound, cudaStream_t st, void* merged_out, int* err_flag) {
+template <int DH, int NG>
+bool launch_t(AttnTc* a, const void* q, int q_rows_cap, int G, const KvView* kv, const RowMeta* const* meta, AttnScratch sc, int rows,
+              int n_heads, int max_ctx, int splits, int keys_bound, cudaStream_t st, void* merged_out, int* err_flag) {
   const CUtensorMap* mq = a->q_map(q, q_rows_cap, n_heads * DH);
-  const CUtensorMap* mk = a->kv_map(kv.k, n_heads, max_ctx, DH);
-  const CUtensorMap* mv = a->kv_map(kv.v, n_heads, max_ctx, DH);
-  if (!mq || !mk || !mv) return false;
-  AttnMaps maps;
+  if (!mq) return false;
+  AttnMaps<NG> maps;
+  AttnParams<NG> prm;
+  if (G > NG) return false;
+  memset(&maps, 0, sizeof maps);
+  memset(&prm, 0, sizeof prm);
   maps.q = *mq;
-  maps.k = *mk;
-  maps.v = *mv;
+  for (int g = 0; g < G; ++g) {
+    const CUtensorMap* mk = a->kv_map(kv[g].k, n_heads, max_ctx, DH);
+    const CUtensorMap* mv = a->kv_map(kv[g].v, n_heads, max_ctx, DH);
+    if (!mk || !mv) return false;
+    maps.k[g] = *mk;
+    maps.v[g] = *mv;
+    prm.meta[g] = meta[g];
+    if (g > 0 && kv[g].k == kv[0].k) prm.same_cache = 1;
+  }
   constexpr int NB = DH / 64;
   constexpr size_t stage = 2 * NB * (size_t)kChunk * 128;
   const int stages = attn_tc_stages(keys_bound, splits, DH);
-  AttnParams prm;
-  prm.meta = meta;
+  prm.nrb = (rows + kRows - 1) / kRows;
+  prm.rpg = rows;
   prm.po = sc.o;
   prm.pml = sc.ml;
   prm.out = (bf16*)merged_out;
@@ -672,7 +695,7 @@ bool launch_t(AttnTc* a, const void* q, int q_rows_cap, KvView kv, const RowMeta
   prm.stages = stages;
   prm.err_flag = err_flag;
   const size_t smem = 1024 + NB * (size_t)kRows * 128 + 2 * (size_t)kRows * 128 + stages * stage;
-  dim3 grid(n_heads, splits, (rows + kRows - 1) / kRows);
+  dim3 grid(n_heads, splits, G * prm.nrb);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(kThreads);
@@ -683,17 +706,17 @@ bool launch_t(AttnTc* a, const void* q, int q_rows_cap, KvView kv, const RowMeta
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   if (merged_out != nullptr) {
-    cudaFuncSetAttribute(tree_attn_tc_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(tree_attn_tc_kernel<DH, true, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     at[1].id = cudaLaunchAttributeClusterDimension;
     at[1].val.clusterDim.x = 1;
     at[1].val.clusterDim.y = splits;
     at[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<DH, true>, maps, prm) == cudaSuccess;
+    return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<DH, true, NG>, maps, prm) == cudaSuccess;
   }
-  cudaFuncSetAttribute(tree_attn_tc_kernel<DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaFuncSetAttribute(tree_attn_tc_kernel<DH, false, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<DH, false>, maps, prm) == cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<DH, false, NG>, maps, prm) == cudaSuccess;
 }
 
 }  // namespace
@@ -707,9 +730,23 @@ bool launch_tree_attention_tc(AttnTc* a, const void* q, int q_rows_cap, KvView k
   if (!a || splits < 1 || (merged_out && splits > 8)) return false;
   if (q_rows_cap < 1) return false;                   // rows of a Q box past the end of the buffer read as zeros
   if (head_dim == 64)
-    return launch_t<64>(a, q, q_rows_cap, kv, meta, sc, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
+    return launch_t<64, 1>(a, q, q_rows_cap, 1, &kv, &meta, sc, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
   if (head_dim == 128)
-    return launch_t<128>(a, q, q_rows_cap, kv, meta, sc, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
+    return launch_t<128, 1>(a, q, q_rows_cap, 1, &kv, &meta, sc, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
+  return false;
+}
+
+// The same for G row groups in ONE launch (grid.z = groups x row blocks): group g's `rows` query rows start at row g * rows of
+// q and of merged_out, read the cache kv[g] and the row table meta[g].  Merged form only (splits <= 8).
+bool launch_tree_attention_tc_groups(AttnTc* a, const void* q, int q_rows_cap, int G, const KvView* kv, const RowMeta* const* meta,
+                                     int rows, int n_heads, int head_dim, int max_ctx, int splits, int keys_bound, cudaStream_t st,
+                                     void* merged_out, int* err_flag) {
+  if (!a || G < 1 || G > kMaxGroups || splits < 1 || splits > 8 || !merged_out || q_rows_cap < G * rows) return false;
+  AttnScratch none = {nullptr, nullptr};
+  if (head_dim == 64)
+    return launch_t<64, kMaxGroups>(a, q, q_rows_cap, G, kv, meta, none, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
+  if (head_dim == 128)
+    return launch_t<128, kMaxGroups>(a, q, q_rows_cap, G, kv, meta, none, rows, n_heads, max_ctx, splits, keys_bound, st, merged_out, err_flag);
   return false;
 }
 

@@ -253,6 +253,60 @@ qkv_rope_kernel(PartialView P, const RowMeta* __restrict__ meta, const float2* _
   }
 }
 
+// The same for G row groups in one launch (blockIdx.z = group): group g's rows start at row g * rpg of P, q and rs and
+// use their own row table, rotary table and cache.
+template <typename T>
+__global__ void __launch_bounds__(256)
+qkv_rope_groups_kernel(PartialView P, RopeGroups gr, T* __restrict__ q, int n_heads, int dh, int max_ctx, RowScale rs) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int g = blockIdx.z, rl = blockIdx.x, r = g * gr.rpg + rl;
+  const RowMeta* meta = gr.meta[g];
+  const float2* rope = gr.rope[g];
+  T* kc = (T*)gr.kc[g];
+  T* vc = (T*)gr.vc[g];
+  const int half = dh >> 1, d = n_heads * dh, quads = half >> 2;
+  const bool live = rl < meta->n_rows;
+  const int slot = meta->slot[rl];
+  const bool store = live && slot >= 0 && slot < max_ctx;
+  const float sc = row_scale(rs, r);
+  for (int idx = blockIdx.y * blockDim.x + threadIdx.x; idx < n_heads * quads; idx += gridDim.y * blockDim.x) {
+    const int h = idx / quads, i = (idx - h * quads) * 4;
+    const float4 cs0 = *reinterpret_cast<const float4*>(rope + rl * half + i);
+    const float4 cs1 = *reinterpret_cast<const float4*>(rope + rl * half + i + 2);
+    const int c0 = h * dh + i, c1 = c0 + half;
+    {
+      float4 a = sum_partials4(P, r, c0), b = sum_partials4(P, r, c1);
+      a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
+      store4(q + (size_t)r * d + c0, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
+                                                 a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
+      store4(q + (size_t)r * d + c1, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
+                                                 b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
+    }
+    if (store) {
+      float4 a = sum_partials4(P, r, d + c0), b = sum_partials4(P, r, d + c1);
+      a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; b.x *= sc; b.y *= sc; b.z *= sc; b.w *= sc;
+      const size_t o = ((size_t)h * max_ctx + slot) * dh + i;
+      store4(kc + o, make_float4(a.x * cs0.x - b.x * cs0.y, a.y * cs0.z - b.y * cs0.w,
+                                 a.z * cs1.x - b.z * cs1.y, a.w * cs1.z - b.w * cs1.w));
+      store4(kc + o + half, make_float4(b.x * cs0.x + a.x * cs0.y, b.y * cs0.z + a.y * cs0.w,
+                                        b.z * cs1.x + a.z * cs1.y, b.w * cs1.z + a.w * cs1.w));
+      float4 v0 = sum_partials4(P, r, 2 * d + c0), v1 = sum_partials4(P, r, 2 * d + c1);
+      store4(vc + o, make_float4(v0.x * sc, v0.y * sc, v0.z * sc, v0.w * sc));
+      store4(vc + o + half, make_float4(v1.x * sc, v1.y * sc, v1.z * sc, v1.w * sc));
+    }
+  }
+}
+
+void launch_qkv_rope_groups(PartialView P, const RopeGroups& gr, void* q, int dtype, int n_heads, int head_dim, int max_ctx,
+                            cudaStream_t st, RowScale rs) {
+  const int items = n_heads * head_dim / 8;
+  const int threads = items >= 128 ? 128 : (items + 31) / 32 * 32;
+  const int gy = (items + threads - 1) / threads;
+  AMPH_DISPATCH(dtype, launch_pdl(qkv_rope_groups_kernel<T>, dim3(gr.rpg, gy, gr.G), dim3(threads), 0, st, P, gr, (T*)q, n_heads,
+                                  head_dim, max_ctx, rs));
+}
+
 void launch_qkv_rope(PartialView P, const RowMeta* meta, const float2* rope, void* q, KvView kv, int dtype,
                      int rows, int n_heads, int head_dim, int max_ctx, cudaStream_t st, RowScale rs) {
   const int items = n_heads * head_dim / 8;
