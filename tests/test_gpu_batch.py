@@ -76,3 +76,22 @@ def test_batched_free_running_steps_are_lossless():
     for b in range(B):
         assert len(got[b]) >= 8 and got[b] == want[b][:len(got[b])]
     model.close()
+
+
+def test_batch_of_four_at_7b_widths():
+    """Four ragged sequences with 64-node trees at the 7B widths (two layers, well-conditioned weights): 256 rows per
+    verification pass, i.e. two 128-row blocks per weight tile in the projections and four row groups per attention and
+    rotary launch at head_dim 128: the launch shapes of the sweep's batch-4 column, at the stated tolerance."""
+    from paper_2406_13170_b200 import Amphista
+    shape = inputs.get_shape("7b").with_(n_layers=2)
+    topo = inputs.make_tree(shape.n_nodes, shape.topk)
+    w_gpu = inputs.make_weights(shape, seed=0, device="cuda:0", init="fan_in")
+    w_cpu = {k: v.cpu() for k, v in w_gpu.items()}
+    lens = (70, 40, 130, 55)
+    model = Amphista(shape, topo, w_gpu, max_batch=4, max_ctx=512)
+    borc = bo.BatchOracle(shape, w_cpu, dtype=torch.float32)
+    reps = run_parity_batch(model, borc, shape, topo, _prompts(shape, lens), 2, 2e-2, 1e-3, None)
+    for r in reps:
+        print(r)
+        assert r.steps == 2
+    model.close()
