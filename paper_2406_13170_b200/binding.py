@@ -19,6 +19,7 @@ AMPH_TOPK_STRIDE = 16
 AMPH_DTYPE_F32, AMPH_DTYPE_BF16 = 0, 1
 AMPH_FLAG_NO_TENSOR_CORE, AMPH_FLAG_NO_GRAPH, AMPH_FLAG_SEPARATE_ROPE = 1, 2, 4
 AMPH_FLAG_SEPARATE_MERGE, AMPH_FLAG_SEPARATE_SWIGLU, AMPH_FLAG_MMA_SYNC_ATTENTION, AMPH_FLAG_NO_SAMPLED_TOKEN = 8, 16, 32, 64
+AMPH_FLAG_CHUNKED_PREFILL, AMPH_FLAG_NO_SIDE_PREFETCH = 128, 256
 STATUS = {0: "AMPH_OK", 1: "AMPH_ERR_INVALID_ARG", 2: "AMPH_ERR_SHAPE", 3: "AMPH_ERR_STATE",
           4: "AMPH_ERR_CAPACITY", 5: "AMPH_ERR_WORKSPACE", 6: "AMPH_ERR_MISSING_WEIGHT",
           7: "AMPH_ERR_CUDA", 8: "AMPH_ERR_TIMEOUT"}

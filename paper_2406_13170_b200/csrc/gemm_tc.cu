@@ -794,6 +794,32 @@ bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, 
   return launch_pdl(tc_gemm_kernel<EPI_ROPE>, dim3(3 * tiles_per_seg, 1), dim3(kThreads), smem, st, pack, prm) == cudaSuccess;
 }
 
+namespace {
+// One thread per CTA asks the TMA unit to bring the first `stages` pipeline stages of every gate / up tile into L2 (stage by
+// stage over all tiles, the order in which the projection's CTAs will ask for them), with the same evict-first policy as the
+// copies themselves: prefetched at normal priority, the weights push the step's L2-resident working set out.
+__global__ void tc_prefetch_pair_kernel(const __grid_constant__ CUtensorMap map, int tiles, int stages, int ks) {
+  if (threadIdx.x != 0) return;
+  const uint64_t pol = l2_evict_first_policy();
+  for (int i = 0; i < stages; ++i)
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x)
+      asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
+                   ::"l"(&map), "r"(0), "r"(t * (kTileM / 2)), "r"(i * ks), "r"(0), "l"(pol) : "memory");
+}
+}  // namespace
+
+bool tc_gemm_prefetch_swiglu(TcGemm* g, const void* w_gate, const void* w_up, int f, int in, size_t budget_bytes, cudaStream_t st) {
+  if (!g || f % (kTileM / 2) || in % (kTileK * kStageKb)) return false;
+  const int stages = (int)(budget_bytes / ((size_t)(f / (kTileM / 2)) * kStageKb * kTileM * kTileK * 2));
+  if (stages <= 0) return false;
+  const bool up_first = (const char*)w_up < (const char*)w_gate;
+  const CUtensorMap* mw = g->get_pair(up_first ? w_up : w_gate, up_first ? w_gate : w_up, f, in, kStageKb);
+  if (!mw) return false;
+  const int max_stages = in / kTileK / kStageKb;
+  tc_prefetch_pair_kernel<<<g->sm_count, 32, 0, st>>>(*mw, f / (kTileM / 2), stages < max_stages ? stages : max_stages, kStageKb);
+  return true;
+}
+
 void tc_gemm_destroy(TcGemm* g) { delete g; }
 
 void tc_gemm_rebind(TcGemm* g, int xb, void* ptr, int rows, int cols, int* err_flag) {

@@ -36,6 +36,10 @@ bool tc_gemm_launch_qkv_rope(TcGemm* g, int xb, const void* wq, const void* wk, 
                              int rows, void* q, KvView kv, const RowMeta* meta, const float2* rope, int max_ctx,
                              const RowScale& rs, cudaStream_t st);
 
+// Asks for the head of every gate / up weight tile (about budget_bytes in all: the first K blocks of all rows of both
+// matrices) to be brought into L2.  A plain launch for a side stream: meant to run while the main stream's kernels leave
+// HBM idle.  Returns false, nothing launched, if the two matrices cannot be described by one tensor map.
+bool tc_gemm_prefetch_swiglu(TcGemm* g, const void* w_gate, const void* w_up, int f, int in, size_t budget_bytes, cudaStream_t st);
 void tc_gemm_destroy(TcGemm* g);
 
 // Points activation buffer `xb` of an existing plan set at another bf16 [rows][cols] buffer and the error flag at

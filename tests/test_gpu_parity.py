@@ -50,8 +50,8 @@ def test_tiny_depth4_tree_and_ragged_prompt():
     model.close()
 
 
-@pytest.mark.parametrize("flags", [1, 0, 4, 8, 16, 32], ids=["plain-kernels", "tensor-core", "separate-rope", "separate-merge",
-                                                            "separate-swiglu", "mma-sync-attention"])
+@pytest.mark.parametrize("flags", [1, 0, 4, 8, 16, 32, 256], ids=["plain-kernels", "tensor-core", "separate-rope", "separate-merge",
+                                                                 "separate-swiglu", "mma-sync-attention", "no-side-prefetch"])
 @pytest.mark.parametrize("planted", [False, True], ids=["natural", "planted"])
 def test_small_bf16_eight_steps(planted, flags):
     """bf16 storage, several 128-row weight tiles, a 32-node tree, a prompt that is not a
