@@ -60,7 +60,7 @@ enum {
                                     * hidden state alone; draft.fc{s} is then [d, d] instead of [d, 2d]            */
   AMPH_FLAG_CHUNKED_PREFILL = 128, /* prefill one chunk of 128 prompt tokens per weight pass instead of four */
   AMPH_FLAG_MMA_SYNC_ATTENTION = 32, /* bf16 tree attention on the warp-level mma.sync kernel instead of the tcgen05 / TMA one */
-  AMPH_FLAG_NO_SIDE_PREFETCH = 256  /* no helper stream: by default (bf16, a stream of the caller's own) every layer forks a small
+  AMPH_FLAG_NO_SIDE_PREFETCH = 256  /* no helper stream: by default (bf16, a stream of the caller's own) every layer of the captured schedule of amph_step forks a small
                                      * kernel onto a second stream, created by amph_init, that pulls the head of the gate / up
                                      * weights into L2 while attention runs; it joins the caller's stream before amph_accept /
                                      * amph_step / amph_prefill return their work to it */

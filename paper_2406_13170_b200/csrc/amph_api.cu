@@ -446,6 +446,10 @@ void fork_prefetch(amph_ctx* ctx, const LayerW& w, int rows) {
   const amph_config& c = ctx->cfg;
   // a gate / up launch of about a full wave (two CTAs per SM) gains nothing: measured +0.3 % at d_ffn = 17920 (280 tiles)
   if (c.d_ffn / 64 > ctx->sm_count * 2 * 13 / 16) return;
+  // only inside the captured schedule of amph_step: launched call by call, the host-side fork and join cost more than the
+  // prefetch gains (measured +95 us per step on the draft / verify / accept path)
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(ctx->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusActive) { cudaGetLastError(); return; }
   if (ctx->fork_used == ctx->fork_ev.size()) { cudaEvent_t e; cudaEventCreateWithFlags(&e, cudaEventDisableTiming); ctx->fork_ev.push_back(e); }
   cudaEvent_t e = ctx->fork_ev[ctx->fork_used++];
   cudaEventRecord(e, ctx->stream);
